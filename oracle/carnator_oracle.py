@@ -1,0 +1,348 @@
+"""CPU oracle for the block-sparse attention path and its connectivity builder.
+
+TEST INFRASTRUCTURE ONLY.  Nothing in the product path imports this module; it
+is called by the tests, by the smoke check and by the CPU-baseline leg of the
+benchmark.  It shares no code with the CUDA path: plain numpy, fp64 unless a
+step says otherwise, no tiling, no online softmax.
+
+What it computes follows the paper's description of historical
+sparse-connectivity reuse (Section 3.3, "Historical Sparse-Connectivity Reuse"
+and "Joint Reuse in Intermediate Layers"; Appendix "Reuse-Scope Implementation
+Details"; Algorithm 1, the last two lines of the denoising loop):
+
+* attention: the target's own Q, K, V; a query attends exactly to the keys
+  whose (query block, key block) pair is present in the historical block mask,
+  or to every key when its query block is flagged target-specific
+  ("recompute").  The result is ordinary softmax attention restricted to that
+  key set, so the oracle is that definition written out.
+* connectivity builder: self-attention is partitioned into query x key blocks
+  and, per head and query block, the smallest set of key blocks that covers a
+  fixed fraction of the attention mass is kept (Appendix "Reuse-Scope
+  Implementation Details").  The graded form estimates block mass from
+  block-pooled Q.K^T scores and selects per row by top-k or by cumulative
+  softmax mass; it is an estimator plus a selection rule, so the oracle takes
+  the steps in order.
+
+Pin status (tests/test_oracle_*.py):
+  attention_rows / attention_full ... pinned (brute force, closed forms, invariants, hand-worked fixture)
+  pooled_scores ..................... pinned (bilinearity identity vs. per-token brute force)
+  forced_blocks ..................... pinned (per-token brute force)
+  select_topk / select_cummass ...... pinned (stable sort, counts, order and minimality invariants)
+  fidelity of the pooled estimator to the true block attention mass: PARITY UNPINNED
+  (the paper prints no mask, density or recall figure; block_mass_exact only reports it).
+"""
+from __future__ import annotations
+
+import math
+from typing import Iterable, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+MODE_TOPK = 0
+MODE_CUMMASS = 1
+
+
+def _widen(bits: np.ndarray) -> np.ndarray:
+    """bf16 bit patterns -> float64, exactly."""
+    u = np.ascontiguousarray(bits, dtype=np.uint16).astype(np.uint32) << np.uint32(16)
+    return u.view(np.float32).astype(np.float64)
+
+
+# ==========================================================================
+# Attention under a block mask  (Section 3.3, Historical Sparse-Connectivity Reuse)
+# ==========================================================================
+def allowed_key_blocks(mask_row: np.ndarray, recompute_flag: int) -> np.ndarray:
+    """Key blocks a query block may attend to: every block if the query block is
+    flagged for recomputation, else the non-zero entries of its mask row."""
+    nkb = mask_row.shape[0]
+    if recompute_flag:
+        return np.arange(nkb)
+    return np.nonzero(mask_row)[0]
+
+
+def attention_rows(Qb: np.ndarray, Kb: np.ndarray, Vb: np.ndarray, N: int,
+                   block_q: int, block_k: int, scale: float,
+                   mask: np.ndarray, recompute: Optional[np.ndarray],
+                   rows: Sequence[Tuple[int, int, int]]):
+    """Masked softmax attention for the listed query blocks.
+
+    Qb, Kb, Vb : uint16 bf16 bits [B, H, >=N, D]
+    mask       : uint8 [B, H, nqb, nkb], non-zero = evaluate the block pair
+    recompute  : uint8 [B, nqb] or None, non-zero = the query block sees every key
+    rows       : (b, h, I) triples
+
+    Returns O [len(rows), block_q, D] and LSE [len(rows), block_q] in fp64; entries
+    of query tokens >= N are NaN.  A query with an empty key set gets O = 0,
+    LSE = -inf.  LSE is the natural log of the sum of exp(scaled scores).
+    """
+    D = Qb.shape[-1]
+    O = np.full((len(rows), block_q, D), np.nan)
+    LSE = np.full((len(rows), block_q), np.nan)
+    cache_key = None
+    K64 = V64 = None
+    for r, (b, h, I) in enumerate(rows):
+        if cache_key != (b, h):
+            K64 = _widen(Kb[b, h, :N])
+            V64 = _widen(Vb[b, h, :N])
+            cache_key = (b, h)
+        i0, i1 = I * block_q, min(N, (I + 1) * block_q)
+        if i0 >= N:
+            continue
+        q = _widen(Qb[b, h, i0:i1])
+        flag = int(recompute[b, I]) if recompute is not None else 0
+        blocks = allowed_key_blocks(mask[b, h, I], flag)
+        cols = [np.arange(J * block_k, min(N, (J + 1) * block_k)) for J in blocks]
+        cols = np.concatenate(cols) if len(cols) else np.zeros((0,), dtype=np.int64)
+        if cols.size == 0:
+            O[r, : i1 - i0] = 0.0
+            LSE[r, : i1 - i0] = -np.inf
+            continue
+        s = scale * (q @ K64[cols].T)                 # s_ij for j in the allowed set
+        m = s.max(axis=1, keepdims=True)
+        p = np.exp(s - m)
+        l = p.sum(axis=1, keepdims=True)
+        O[r, : i1 - i0] = (p @ V64[cols]) / l
+        LSE[r, : i1 - i0] = (m + np.log(l))[:, 0]
+    return O, LSE
+
+
+def attention_full(Qb, Kb, Vb, N, block_q, block_k, scale, mask, recompute=None):
+    """All query blocks of all heads: O [B, H, N, D], LSE [B, H, N] in fp64."""
+    B, H = Qb.shape[0], Qb.shape[1]
+    D = Qb.shape[-1]
+    nqb = -(-N // block_q)
+    rows = [(b, h, I) for b in range(B) for h in range(H) for I in range(nqb)]
+    Or, Lr = attention_rows(Qb, Kb, Vb, N, block_q, block_k, scale, mask, recompute, rows)
+    O = Or.reshape(B, H, nqb * block_q, D)[:, :, :N]
+    L = Lr.reshape(B, H, nqb * block_q)[:, :, :N]
+    return O, L
+
+
+def dense_bruteforce(Qb, Kb, Vb, N, block_q, block_k, scale, mask, recompute=None):
+    """Second, independent statement of the same definition, for tiny inputs only.
+
+    Materialises the N x N score matrix of each head with -inf at every
+    disallowed (query, key) pair and evaluates softmax one query at a time with
+    Python scalars.  Used only to check attention_rows / attention_full.
+    """
+    B, H = Qb.shape[0], Qb.shape[1]
+    D = Qb.shape[-1]
+    O = np.zeros((B, H, N, D))
+    LSE = np.zeros((B, H, N))
+    for b in range(B):
+        for h in range(H):
+            q = _widen(Qb[b, h, :N])
+            k = _widen(Kb[b, h, :N])
+            v = _widen(Vb[b, h, :N])
+            S = np.full((N, N), -np.inf)
+            for i in range(N):
+                I = i // block_q
+                dense = recompute is not None and recompute[b, I] != 0
+                for j in range(N):
+                    if dense or mask[b, h, I, j // block_k] != 0:
+                        acc = 0.0
+                        for d in range(D):
+                            acc += q[i, d] * k[j, d]
+                        S[i, j] = scale * acc
+            for i in range(N):
+                mx = max(S[i])
+                if mx == -np.inf:
+                    LSE[b, h, i] = -np.inf
+                    continue
+                den = 0.0
+                num = np.zeros(D)
+                for j in range(N):
+                    if S[i, j] != -np.inf:
+                        e = math.exp(S[i, j] - mx)
+                        den += e
+                        num += e * v[j]
+                O[b, h, i] = num / den
+                LSE[b, h, i] = mx + math.log(den)
+    return O, LSE
+
+
+# ==========================================================================
+# Connectivity builder  (Appendix "Reuse-Scope Implementation Details")
+# ==========================================================================
+def pooled_means(Xb_head: np.ndarray, N: int, block: int) -> np.ndarray:
+    """Step 1: mean of each block's VALID token rows, fp64 accumulate -> fp32.  [nb, D] float32."""
+    nb = -(-N // block)
+    X = _widen(Xb_head[:N])
+    out = np.zeros((nb, X.shape[1]), dtype=np.float32)
+    for I in range(nb):
+        seg = X[I * block: min(N, (I + 1) * block)]
+        out[I] = (seg.sum(axis=0) / seg.shape[0]).astype(np.float32)
+    return out
+
+
+def pooled_scores(Qb_head, Kb_head, N, block_q, block_k, scale) -> np.ndarray:
+    """Step 2: S~[I, J] = fp32(scale * <q_bar_I, k_bar_J>), fp64 accumulate.  This fp32
+    value is 'the pooled score' that selection and the tolerance band refer to."""
+    qbar = pooled_means(Qb_head, N, block_q).astype(np.float64)
+    kbar = pooled_means(Kb_head, N, block_k).astype(np.float64)
+    return (np.float64(np.float32(scale)) * (qbar @ kbar.T)).astype(np.float32)
+
+
+def forced_blocks(N, n_text, T, Hg, Wg, block_q, block_k, window_frames, text_dense) -> np.ndarray:
+    """Step 3: bool [nqb, nkb], blocks kept regardless of score.
+
+    text_dense: a query block holding a text token keeps every key block, and every
+    key block holding a text token is kept by every query block.
+    window_frames = r >= 0: a query block whose video tokens span frames f_lo..f_hi
+    keeps every key block holding a video token of frames [f_lo - r, f_hi + r].
+    Token order: text first, then video flattened frame-major.
+    """
+    nqb, nkb = -(-N // block_q), -(-N // block_k)
+    hw = Hg * Wg
+    F = np.zeros((nqb, nkb), dtype=bool)
+
+    def frames_of(block, I):
+        lo, hi = I * block, min(N, (I + 1) * block) - 1
+        lo = max(lo, n_text)
+        if hi < lo:
+            return None
+        return (lo - n_text) // hw, (hi - n_text) // hw
+
+    kf = [frames_of(block_k, J) for J in range(nkb)]
+    for I in range(nqb):
+        if text_dense and n_text > 0 and I * block_q < n_text:
+            F[I, :] = True
+            continue
+        if text_dense and n_text > 0:
+            for J in range(nkb):
+                if J * block_k < n_text:
+                    F[I, J] = True
+        if window_frames >= 0:
+            qf = frames_of(block_q, I)
+            if qf is not None:
+                lo = max(0, qf[0] - window_frames)
+                hi = min(T - 1, qf[1] + window_frames)
+                for J in range(nkb):
+                    if kf[J] is not None and kf[J][0] <= hi and kf[J][1] >= lo:
+                        F[I, J] = True
+    return F
+
+
+def topk_count(keep_ratio: float, n_candidates: int) -> int:
+    """k = ceil(ratio * n - 1e-6) clamped to [1, n] (0 when there is no candidate).
+    The ratio is taken at fp32 precision, as it travels through the C struct."""
+    if n_candidates <= 0:
+        return 0
+    k = math.ceil(float(np.float32(keep_ratio)) * n_candidates - 1e-6)
+    return max(1, min(n_candidates, k))
+
+
+def _descending_stable(scores: np.ndarray, idx: np.ndarray) -> np.ndarray:
+    """idx reordered by score descending; equal scores keep ascending block index."""
+    order = np.argsort(-scores[idx].astype(np.float64), kind="stable")
+    return idx[order]
+
+
+def select_topk(scores_row: np.ndarray, forced_row: np.ndarray, keep_ratio: float,
+                count_includes_forced: int):
+    """Step 4.  Returns (keep bool[nkb], theta) with theta the score of the last block
+    admitted by score (NaN if none was)."""
+    nkb = scores_row.shape[0]
+    keep = forced_row.copy()
+    free = np.nonzero(~forced_row)[0]
+    if count_includes_forced:
+        k = topk_count(keep_ratio, nkb)
+        n_admit = max(0, k - int(forced_row.sum()))
+    else:
+        n_admit = topk_count(keep_ratio, free.size)
+    n_admit = min(n_admit, free.size)
+    theta = np.float32(np.nan)
+    if n_admit > 0:
+        ranked = _descending_stable(scores_row, free)
+        keep[ranked[:n_admit]] = True
+        theta = scores_row[ranked[n_admit - 1]]
+    return keep, theta
+
+
+def select_cummass(scores_row: np.ndarray, forced_row: np.ndarray, mass: float):
+    """Step 5.  p = softmax over all key blocks of the pooled scores (fp64); non-forced
+    blocks are admitted in descending score order until the kept mass (forced blocks
+    included) reaches ``mass`` -- the smallest descending prefix that covers it."""
+    s = scores_row.astype(np.float64)
+    p = np.exp(s - s.max())
+    p = p / p.sum()
+    keep = forced_row.copy()
+    free = np.nonzero(~forced_row)[0]
+    ranked = _descending_stable(scores_row, free)
+    target = float(np.float32(mass))
+    running = float(p[forced_row].sum())
+    theta = np.float32(np.nan)
+    for J in ranked:
+        if running >= target:
+            break
+        keep[J] = True
+        running += p[J]
+        theta = scores_row[J]
+    return keep, theta
+
+
+def build_connectivity(Qb, Kb, N, n_text, T, Hg, Wg, block_q, block_k, scale,
+                       mode=MODE_TOPK, keep_ratio=0.25, mass=0.9, window_frames=-1,
+                       text_dense=0, count_includes_forced=1,
+                       heads: Optional[Iterable[Tuple[int, int]]] = None):
+    """Steps 1-6 for every (or the listed) head.
+
+    Returns mask uint8 [B, H, nqb, nkb], scores float32 [B, H, nqb, nkb],
+    theta float32 [B, H, nqb] (NaN where no block was admitted by score) and the
+    forced-block table bool [nqb, nkb].  Heads not listed stay zero.
+    """
+    B, H = Qb.shape[0], Qb.shape[1]
+    nqb, nkb = -(-N // block_q), -(-N // block_k)
+    F = forced_blocks(N, n_text, T, Hg, Wg, block_q, block_k, window_frames, text_dense)
+    mask = np.zeros((B, H, nqb, nkb), dtype=np.uint8)
+    scores = np.zeros((B, H, nqb, nkb), dtype=np.float32)
+    theta = np.full((B, H, nqb), np.nan, dtype=np.float32)
+    todo = list(heads) if heads is not None else [(b, h) for b in range(B) for h in range(H)]
+    for (b, h) in todo:
+        S = pooled_scores(Qb[b, h], Kb[b, h], N, block_q, block_k, scale)
+        scores[b, h] = S
+        for I in range(nqb):
+            if mode == MODE_TOPK:
+                keep, th = select_topk(S[I], F[I], keep_ratio, count_includes_forced)
+            elif mode == MODE_CUMMASS:
+                keep, th = select_cummass(S[I], F[I], mass)
+            else:
+                raise ValueError("unknown selection mode")
+            mask[b, h, I] = keep
+            theta[b, h, I] = th
+    return mask, scores, theta, F
+
+
+def block_mass_exact(Qb_head, Kb_head, N, block_q, block_k, scale) -> np.ndarray:
+    """The paper's literal quantity, for reporting only (tiny inputs): the share of a
+    query block's softmax attention mass that falls in each key block, averaged over
+    the block's queries.  [nqb, nkb] fp64, rows sum to 1."""
+    q = _widen(Qb_head[:N])
+    k = _widen(Kb_head[:N])
+    s = scale * (q @ k.T)
+    p = np.exp(s - s.max(axis=1, keepdims=True))
+    p /= p.sum(axis=1, keepdims=True)
+    nqb, nkb = -(-N // block_q), -(-N // block_k)
+    out = np.zeros((nqb, nkb))
+    for I in range(nqb):
+        rows = p[I * block_q: min(N, (I + 1) * block_q)]
+        for J in range(nkb):
+            out[I, J] = rows[:, J * block_k: min(N, (J + 1) * block_k)].sum() / rows.shape[0]
+    return out
+
+
+# ==========================================================================
+# counting helpers used by tests and the benchmark
+# ==========================================================================
+def computed_tile_flops(N, D, block_q, block_k, mask, recompute=None) -> float:
+    """4 * rows_valid * cols_valid * D summed over evaluated block pairs (all heads)."""
+    B, H, nqb, nkb = mask.shape
+    rq = np.minimum(block_q, N - np.arange(nqb) * block_q).astype(np.float64)
+    ck = np.minimum(block_k, N - np.arange(nkb) * block_k).astype(np.float64)
+    total = 0.0
+    for b in range(B):
+        eff = mask[b] != 0
+        if recompute is not None:
+            eff = eff | (recompute[b] != 0)[None, :, None]
+        total += 4.0 * D * float(np.einsum("hij,i,j->", eff.astype(np.float64), rq, ck))
+    return total
