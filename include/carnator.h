@@ -1,0 +1,210 @@
+/*
+ * carnator.h -- C ABI of the block-sparse attention hot path (CUDA, sm_100a).
+ *
+ * The library executes one self-attention layer of a video diffusion
+ * transformer the way the paper's cross-request reuse does on a cache hit:
+ * the target request's own Q, K and V are used, but only the (query block,
+ * key block) pairs recorded in a historical request's block-connectivity mask
+ * are evaluated; query blocks flagged as target-specific are evaluated
+ * densely.  A companion call builds such a mask from block-pooled Q.K^T scores
+ * when a request's computation is written into the cache.
+ *
+ * General conventions (every entry point):
+ *   - Unless a parameter is documented as a HOST pointer, every data pointer is
+ *     a DEVICE pointer owned by the caller.  The library never allocates or
+ *     frees device memory; scratch space is passed in as a workspace whose size
+ *     the *_workspace_bytes queries return.
+ *   - Calls are asynchronous on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the default stream).  Only carnator_query_status and the *_host calls
+ *     synchronise.
+ *   - Arguments are validated on the host before any launch.  A failed call
+ *     launches nothing and returns an error code; nothing aborts or throws.
+ *   - Q, K, V, O are bf16 with the head dimension contiguous; the element
+ *     strides of the (batch, head, token) axes are given in the shape record and
+ *     must be multiples of 8 elements (16 bytes); base pointers 16-byte aligned.
+ *   - Token order: text tokens first (n_text of them), then video tokens
+ *     flattened frame-major (t, then grid row, then grid column).  Blocks are
+ *     contiguous runs of block_q / block_k tokens of that order; the last block
+ *     may be partial.  Buffers may hold more than N rows; rows >= N are never
+ *     read as keys and never written.
+ *   - Mask bytes and recompute bytes: non-zero = keep / recompute.
+ *   - Attention is bidirectional softmax attention; LSE is the natural log of
+ *     the sum of exp(scaled scores) over the keys a query sees.  A query that
+ *     sees no key gets O = 0 and LSE = -inf.
+ *   - There is no CPU fallback: on a machine without an sm_100 device the
+ *     compute calls return CARNATOR_ERR_UNSUPPORTED.
+ */
+#ifndef CARNATOR_H_
+#define CARNATOR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum carnator_status {
+    CARNATOR_OK = 0,
+    CARNATOR_ERR_INVALID_ARG = 1,   /* NULL pointer, non-positive size, misaligned pointer or stride, n_text + T*Hg*Wg != N */
+    CARNATOR_ERR_UNSUPPORTED = 2,   /* D not in {64,128}, block size not in {64,128}, too many key blocks, no sm_100 device */
+    CARNATOR_ERR_WORKSPACE = 3,     /* workspace NULL, misaligned (256 B) or smaller than the matching *_workspace_bytes */
+    CARNATOR_ERR_CUDA = 4,          /* a CUDA runtime / driver call failed; see carnator_last_cuda_error */
+    CARNATOR_ERR_DEVICE_TIMEOUT = 5,/* a bounded wait inside a kernel expired; the kernel drained and returned */
+    CARNATOR_ERR_DEVICE_CHECK = 6   /* a device-side consistency check failed (malformed compacted lists) */
+} carnator_status;
+
+/* Which attention kernel executes the compacted lists. */
+enum {
+    CARNATOR_IMPL_AUTO = 0,      /* tcgen05 kernel where it supports the shape, else the portable kernel */
+    CARNATOR_IMPL_PORTABLE = 1,  /* mma.sync kernel: any supported shape */
+    CARNATOR_IMPL_TCGEN05 = 2    /* TMA + tcgen05/TMEM kernel: block_q = block_k = 128; else CARNATOR_ERR_UNSUPPORTED */
+};
+
+/* Problem description shared by all calls. */
+typedef struct carnator_shape {
+    int32_t B, H, N, D;             /* batch, heads, valid tokens per head, head dimension (64 or 128) */
+    int32_t n_text, T, Hg, Wg;      /* n_text + T*Hg*Wg == N; latent grid T x Hg x Wg */
+    int32_t block_q, block_k;       /* 64 or 128 */
+    int64_t q_stride[3];            /* element strides of (batch, head, token) for Q; head dim has stride 1 */
+    int64_t k_stride[3];
+    int64_t v_stride[3];
+    int64_t o_stride[3];
+    float   softmax_scale;          /* <= 0 selects 1/sqrt(D) */
+    int32_t attn_impl;              /* CARNATOR_IMPL_* */
+} carnator_shape;
+
+/* Selection rule of the connectivity builder. */
+enum { CARNATOR_MODE_TOPK = 0, CARNATOR_MODE_CUMMASS = 1 };
+
+typedef struct carnator_build_params {
+    int32_t mode;                   /* CARNATOR_MODE_TOPK: keep_ratio; CARNATOR_MODE_CUMMASS: mass */
+    float   keep_ratio;             /* TOPK: k = clamp(ceil(keep_ratio * n - 1e-6), 1, n) over the n candidates of a row */
+    float   mass;                   /* CUMMASS: fraction of the row's pooled-softmax mass to cover, in (0, 1] */
+    int32_t window_frames;          /* -1: none; r >= 0: key blocks touching frames [f_lo - r, f_hi + r] of the query block are always kept */
+    int32_t text_dense;             /* 1: blocks holding a text token are dense rows and dense columns */
+    int32_t count_includes_forced;  /* TOPK: 1: k counts the always-kept blocks; 0: k applies to the other candidates only */
+} carnator_build_params;
+
+/* ------------------------------------------------------------------------
+ * Connectivity builder (cache-write side).
+ *
+ * Paper: Appendix "Reuse-Scope Implementation Details" -- self-attention is
+ * partitioned into query x key blocks and, per head and query block, the
+ * smallest set of key blocks covering a fixed fraction of the attention mass is
+ * kept as a binary mask.  This call estimates block mass from block-pooled
+ * scores: q_bar_I / k_bar_J = mean of the block's valid token rows (fp32),
+ * S[I,J] = scale * <q_bar_I, k_bar_J> (fp32), then per row either the k best
+ * blocks (ties: lower key-block index first) or the shortest descending prefix
+ * whose softmax mass over the row reaches `mass`, in both cases together with
+ * the always-kept blocks (frame window, text rows / columns).
+ *
+ *   Q, K   device, bf16 [B,H,>=N,D] with the strides of `shape`
+ *   mask   device, uint8 [B,H,nqb,nkb] contiguous, written (1 = keep, 0 = drop)
+ *   pooled_scores_opt  device, fp32 [B,H,nqb,nkb] contiguous or NULL; when given it
+ *          receives S (and replaces the score area of the workspace)
+ *   ws     device workspace, 256-byte aligned, >= carnator_build_workspace_bytes
+ * Limits: nkb <= 4096.
+ * ------------------------------------------------------------------------ */
+size_t carnator_build_workspace_bytes(const carnator_shape* shape, const carnator_build_params* params);
+
+carnator_status carnator_build_connectivity(const void* Q, const void* K,
+                                            const carnator_shape* shape,
+                                            const carnator_build_params* params,
+                                            uint8_t* mask, float* pooled_scores_opt,
+                                            void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Sparse attention under a reused mask (cache-hit side).
+ *
+ * Paper: Section 3.3, "Historical Sparse-Connectivity Reuse" (the target's Q, K,
+ * V are recomputed; the historical block structure decides which query-key
+ * interactions are evaluated) and "Joint Reuse in Intermediate Layers" /
+ * Algorithm 1 (target-specific query blocks are recomputed); latency accounting
+ * of mask / index lookups: Appendix "Latency Accounting".
+ *
+ * Query block I of head (b,h) attends to every key of key block J iff
+ * recompute_rows[b,I] != 0 or mask[b,h,I,J] != 0.
+ *
+ *   Q, K, V  device, bf16, strides of `shape`
+ *   mask     device, uint8 [B,H,nqb,nkb] contiguous (read only)
+ *   recompute_rows  device, uint8 [B,nqb] contiguous, or NULL for "none"
+ *   O        device, bf16, strides o_stride; rows < N written
+ *   LSE      device, fp32 [B,H,N] contiguous
+ *   ws       device workspace, 256-byte aligned, >= carnator_attn_workspace_bytes
+ *
+ * carnator_sparse_attn = carnator_compact_mask + carnator_sparse_attn_compacted.
+ * The split lets a caller compact a mask once and reuse the lists (a mask belongs
+ * to one denoising step, guidance branch and layer and is the same for every
+ * request that reuses that cache entry).  The workspace then carries the lists
+ * between the two calls and must not be modified in between.
+ *
+ * carnator_compact_mask writes, per (b,h,I), the ascending list of key blocks to
+ * evaluate and its length, and per (b,h) an execution order of the query blocks
+ * (longest list first).
+ * ------------------------------------------------------------------------ */
+size_t carnator_attn_workspace_bytes(const carnator_shape* shape);
+
+carnator_status carnator_compact_mask(const uint8_t* mask, const uint8_t* recompute_rows,
+                                      const carnator_shape* shape,
+                                      void* ws, size_t ws_bytes, void* stream);
+
+carnator_status carnator_sparse_attn_compacted(const void* Q, const void* K, const void* V,
+                                               const carnator_shape* shape,
+                                               void* O, float* LSE,
+                                               void* ws, size_t ws_bytes, void* stream);
+
+carnator_status carnator_sparse_attn(const void* Q, const void* K, const void* V,
+                                     const uint8_t* mask, const uint8_t* recompute_rows,
+                                     const carnator_shape* shape,
+                                     void* O, float* LSE,
+                                     void* ws, size_t ws_bytes, void* stream);
+
+/* Number of evaluated (query block, key block) pairs after compaction, summed over
+ * all heads.  Synchronises `stream`.  *tiles is a HOST pointer. */
+carnator_status carnator_compacted_tiles(const carnator_shape* shape, const void* ws, size_t ws_bytes,
+                                         void* stream, int64_t* tiles);
+
+/* ------------------------------------------------------------------------
+ * Host-buffer forms of the two calls (end-to-end use and measurement).
+ * Q/K/V/mask/recompute_rows/O/LSE/pooled scores are HOST pointers (pinned memory
+ * for full copy speed) laid out contiguously: Q,K,V,O [B,H,N,D] bf16 (the strides
+ * in `shape` are ignored), LSE [B,H,N], mask [B,H,nqb,nkb], recompute_rows [B,nqb].
+ * `arena` is a DEVICE buffer of at least carnator_*_host_arena_bytes that holds
+ * the device copies and the workspace.  The calls copy in, run, copy out and
+ * synchronise `stream` before returning.
+ * ------------------------------------------------------------------------ */
+size_t carnator_attn_host_arena_bytes(const carnator_shape* shape);
+
+carnator_status carnator_sparse_attn_host(const void* Q, const void* K, const void* V,
+                                          const uint8_t* mask, const uint8_t* recompute_rows,
+                                          const carnator_shape* shape,
+                                          void* O, float* LSE,
+                                          void* arena, size_t arena_bytes, void* stream);
+
+size_t carnator_build_host_arena_bytes(const carnator_shape* shape, const carnator_build_params* params);
+
+carnator_status carnator_build_connectivity_host(const void* Q, const void* K,
+                                                 const carnator_shape* shape,
+                                                 const carnator_build_params* params,
+                                                 uint8_t* mask,
+                                                 void* arena, size_t arena_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * Status and diagnostics.
+ * carnator_query_status synchronises `stream` and returns the status word that
+ * kernels of earlier calls on this workspace may have set (CARNATOR_OK,
+ * CARNATOR_ERR_DEVICE_TIMEOUT or CARNATOR_ERR_DEVICE_CHECK), then clears it.
+ * carnator_kernel_launches returns how many kernels this library has launched in
+ * the calling process so far (monotone counter).
+ * ------------------------------------------------------------------------ */
+carnator_status carnator_query_status(void* ws, void* stream);
+const char*     carnator_status_string(carnator_status s);
+const char*     carnator_last_cuda_error(void);
+int64_t         carnator_kernel_launches(void);
+int32_t         carnator_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CARNATOR_H_ */

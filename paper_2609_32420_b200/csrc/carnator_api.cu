@@ -1,0 +1,462 @@
+// C-ABI entry points of libcarnator: argument validation, workspace layout, kernel launches.
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+
+#include "carnator.h"
+#include "common.cuh"
+#include "builder.cuh"
+#include "compact.cuh"
+#include "attn_portable.cuh"
+#include "attn_tcgen05.cuh"
+
+using namespace carnator;
+
+namespace {
+
+std::atomic<long long> g_launches{0};
+thread_local char g_cuda_error[256] = "";
+
+carnator_status cuda_fail(cudaError_t e, const char* where) {
+    snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", where, cudaGetErrorString(e));
+    return CARNATOR_ERR_CUDA;
+}
+
+#define CUDA_TRY(expr)                                              \
+    do {                                                            \
+        cudaError_t e__ = (expr);                                   \
+        if (e__ != cudaSuccess) return cuda_fail(e__, #expr);       \
+    } while (0)
+
+#define LAUNCH_CHECK(name)                                          \
+    do {                                                            \
+        g_launches.fetch_add(1, std::memory_order_relaxed);         \
+        cudaError_t e__ = cudaGetLastError();                       \
+        if (e__ != cudaSuccess) return cuda_fail(e__, name);        \
+    } while (0)
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bool strides_ok(const int64_t s[3]) {
+    return s[0] >= 0 && s[1] >= 0 && s[2] > 0 && s[0] % 8 == 0 && s[1] % 8 == 0 && s[2] % 8 == 0;
+}
+
+carnator_status check_shape(const carnator_shape* s, bool need_v_o) {
+    if (!s) return CARNATOR_ERR_INVALID_ARG;
+    if (s->B <= 0 || s->H <= 0 || s->N <= 0 || s->D <= 0) return CARNATOR_ERR_INVALID_ARG;
+    if (s->n_text < 0 || s->T < 0 || s->Hg < 0 || s->Wg < 0) return CARNATOR_ERR_INVALID_ARG;
+    if (int64_t(s->n_text) + int64_t(s->T) * s->Hg * s->Wg != int64_t(s->N)) return CARNATOR_ERR_INVALID_ARG;
+    if (s->block_q <= 0 || s->block_k <= 0) return CARNATOR_ERR_INVALID_ARG;
+    if (s->D != 64 && s->D != 128) return CARNATOR_ERR_UNSUPPORTED;
+    if ((s->block_q != 64 && s->block_q != 128) || (s->block_k != 64 && s->block_k != 128)) return CARNATOR_ERR_UNSUPPORTED;
+    if (!strides_ok(s->q_stride) || !strides_ok(s->k_stride)) return CARNATOR_ERR_INVALID_ARG;
+    if (s->q_stride[2] < s->D || s->k_stride[2] < s->D) return CARNATOR_ERR_INVALID_ARG;
+    if (need_v_o) {
+        if (!strides_ok(s->v_stride) || !strides_ok(s->o_stride)) return CARNATOR_ERR_INVALID_ARG;
+        if (s->v_stride[2] < s->D || s->o_stride[2] < s->D) return CARNATOR_ERR_INVALID_ARG;
+    }
+    if (s->attn_impl < CARNATOR_IMPL_AUTO || s->attn_impl > CARNATOR_IMPL_TCGEN05) return CARNATOR_ERR_INVALID_ARG;
+    if (std::isnan(s->softmax_scale) || std::isinf(s->softmax_scale)) return CARNATOR_ERR_INVALID_ARG;
+    return CARNATOR_OK;
+}
+
+carnator_status check_params(const carnator_build_params* p) {
+    if (!p) return CARNATOR_ERR_INVALID_ARG;
+    if (p->mode != CARNATOR_MODE_TOPK && p->mode != CARNATOR_MODE_CUMMASS) return CARNATOR_ERR_INVALID_ARG;
+    if (p->mode == CARNATOR_MODE_TOPK && !(p->keep_ratio > 0.f && p->keep_ratio <= 1.f)) return CARNATOR_ERR_INVALID_ARG;
+    if (p->mode == CARNATOR_MODE_CUMMASS && !(p->mass > 0.f && p->mass <= 1.f)) return CARNATOR_ERR_INVALID_ARG;
+    if (p->window_frames < -1) return CARNATOR_ERR_INVALID_ARG;
+    return CARNATOR_OK;
+}
+
+// The device must be sm_100 (the kernels are built for sm_100a only).
+carnator_status check_device() {
+    static thread_local int cached_dev = -1;
+    static thread_local carnator_status cached = CARNATOR_OK;
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) { cudaGetLastError(); snprintf(g_cuda_error, sizeof(g_cuda_error), "cudaGetDevice: %s", cudaGetErrorString(e)); return CARNATOR_ERR_UNSUPPORTED; }
+    if (dev == cached_dev) return cached;
+    int major = 0;
+    e = cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev);
+    if (e != cudaSuccess) { cudaGetLastError(); return CARNATOR_ERR_UNSUPPORTED; }
+    cached_dev = dev;
+    cached = (major == 10) ? CARNATOR_OK : CARNATOR_ERR_UNSUPPORTED;
+    return cached;
+}
+
+float effective_scale(const carnator_shape* s) {
+    return s->softmax_scale > 0.f ? s->softmax_scale : 1.0f / sqrtf(float(s->D));
+}
+
+int next_pow2(int x) { int p = 1; while (p < x) p <<= 1; return p; }
+
+int topk_count_host(float ratio, int n) {
+    if (n <= 0) return 0;
+    double x = double(ratio) * double(n) - 1e-6;
+    int k = int(std::ceil(x));
+    return k < 1 ? 1 : (k > n ? n : k);
+}
+
+template <typename K>
+carnator_status allow_smem(K kernel, size_t bytes) {
+    CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(bytes)));
+    return CARNATOR_OK;
+}
+
+}  // namespace
+
+// ------------------------------------------------------------------------------------------------
+// builder
+// ------------------------------------------------------------------------------------------------
+extern "C" size_t carnator_build_workspace_bytes(const carnator_shape* s, const carnator_build_params* p) {
+    if (check_shape(s, false) != CARNATOR_OK || check_params(p) != CARNATOR_OK) return 0;
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    return build_ws_layout(nullptr, s->B, s->H, nqb, nkb, s->D).bytes;
+}
+
+extern "C" carnator_status carnator_build_connectivity(const void* Q, const void* K, const carnator_shape* s,
+                                                       const carnator_build_params* p, uint8_t* mask,
+                                                       float* pooled_scores_opt, void* ws, size_t ws_bytes,
+                                                       void* stream_) {
+    carnator_status st = check_shape(s, false);
+    if (st != CARNATOR_OK) return st;
+    st = check_params(p);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !mask) return CARNATOR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16)) return CARNATOR_ERR_INVALID_ARG;
+    if (pooled_scores_opt && !aligned(pooled_scores_opt, 16)) return CARNATOR_ERR_INVALID_ARG;
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    if (nkb > kMaxKeyBlocksBuilder) return CARNATOR_ERR_UNSUPPORTED;
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    BuildWs w = build_ws_layout(ws, s->B, s->H, nqb, nkb, s->D);
+    if (ws_bytes < w.bytes) return CARNATOR_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    float* scores = pooled_scores_opt ? pooled_scores_opt : w.scores;
+
+    CUDA_TRY(cudaMemsetAsync(w.hdr, 0, sizeof(WsHeader), stream));
+
+    // M1
+    PoolArgs pa;
+    pa.X[0] = static_cast<const __nv_bfloat16*>(Q);
+    pa.X[1] = static_cast<const __nv_bfloat16*>(K);
+    for (int i = 0; i < 3; ++i) { pa.stride[0][i] = s->q_stride[i]; pa.stride[1][i] = s->k_stride[i]; }
+    pa.block[0] = s->block_q; pa.block[1] = s->block_k;
+    pa.nb[0] = nqb; pa.nb[1] = nkb;
+    pa.out[0] = w.qbar; pa.out[1] = w.kbar;
+    pa.N = s->N; pa.H = s->H;
+    {
+        dim3 grid(nqb > nkb ? nqb : nkb, s->H, 2 * s->B);
+        if (s->D == 128) pool_kernel<128><<<grid, 256, 0, stream>>>(pa);
+        else pool_kernel<64><<<grid, 256, 0, stream>>>(pa);
+        LAUNCH_CHECK("pool_kernel");
+    }
+    // M2
+    {
+        dim3 grid(ceil_div(nkb, 64), ceil_div(nqb, 64), s->B * s->H);
+        const float scale = effective_scale(s);
+        if (s->D == 128) score_kernel<128><<<grid, 256, 0, stream>>>(w.qbar, w.kbar, scores, nqb, nkb, scale);
+        else score_kernel<64><<<grid, 256, 0, stream>>>(w.qbar, w.kbar, scores, nqb, nkb, scale);
+        LAUNCH_CHECK("score_kernel");
+    }
+    // M3
+    {
+        SelectArgs sa;
+        sa.scores = scores; sa.mask = mask;
+        sa.nqb = nqb; sa.nkb = nkb; sa.npad = next_pow2(nkb); sa.H = s->H;
+        sa.mode = p->mode; sa.keep_ratio = p->keep_ratio; sa.mass = p->mass;
+        sa.count_includes_forced = p->count_includes_forced;
+        sa.k_all = topk_count_host(p->keep_ratio, nkb);
+        sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
+        sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
+        size_t smem = size_t(sa.npad) * 8 * (p->mode == CARNATOR_MODE_CUMMASS ? 2 : 1) + ((nkb + 15) & ~15);
+        st = allow_smem(select_kernel, 72 * 1024);
+        if (st != CARNATOR_OK) return st;
+        dim3 grid(nqb, s->H, s->B);
+        select_kernel<<<grid, 256, smem, stream>>>(sa);
+        LAUNCH_CHECK("select_kernel");
+    }
+    return CARNATOR_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// compaction + attention
+// ------------------------------------------------------------------------------------------------
+extern "C" size_t carnator_attn_workspace_bytes(const carnator_shape* s) {
+    if (check_shape(s, true) != CARNATOR_OK) return 0;
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    return attn_ws_layout(nullptr, s->B, s->H, nqb, nkb).bytes;
+}
+
+static carnator_status attn_ws_check(const carnator_shape* s, void* ws, size_t ws_bytes, AttnWs* out) {
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    *out = attn_ws_layout(ws, s->B, s->H, nqb, nkb);
+    if (ws_bytes < out->bytes) return CARNATOR_ERR_WORKSPACE;
+    return CARNATOR_OK;
+}
+
+extern "C" carnator_status carnator_compact_mask(const uint8_t* mask, const uint8_t* recompute_rows,
+                                                 const carnator_shape* s, void* ws, size_t ws_bytes, void* stream_) {
+    carnator_status st = check_shape(s, true);
+    if (st != CARNATOR_OK) return st;
+    if (!mask) return CARNATOR_ERR_INVALID_ARG;
+    AttnWs w;
+    st = attn_ws_check(s, ws, ws_bytes, &w);
+    if (st != CARNATOR_OK) return st;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    if (nqb > 12000) return CARNATOR_ERR_UNSUPPORTED;   // order kernel keeps one head's counts in shared memory
+    CUDA_TRY(cudaMemsetAsync(w.hdr, 0, sizeof(WsHeader), stream));
+    const int rows = s->B * s->H * nqb;
+    compact_rows_kernel<<<ceil_div(rows, 8), 256, 0, stream>>>(mask, recompute_rows, s->B, s->H, nqb, nkb, w.counts, w.lists);
+    LAUNCH_CHECK("compact_rows_kernel");
+    order_rows_kernel<<<s->B * s->H, 256, size_t(nqb) * 4, stream>>>(w.counts, nqb, w.order, w.hdr);
+    LAUNCH_CHECK("order_rows_kernel");
+    return CARNATOR_OK;
+}
+
+template <int D, int BQ>
+static carnator_status launch_portable(const AttnArgs& a, cudaStream_t stream) {
+    using C = PortableCfg<D, BQ>;
+    carnator_status st = allow_smem(attn_portable_kernel<D, BQ>, C::smem_bytes);
+    if (st != CARNATOR_OK) return st;
+    dim3 grid(a.nqb, a.H, a.B);
+    attn_portable_kernel<D, BQ><<<grid, C::NT, C::smem_bytes, stream>>>(a);
+    LAUNCH_CHECK("attn_portable_kernel");
+    return CARNATOR_OK;
+}
+
+extern "C" carnator_status carnator_sparse_attn_compacted(const void* Q, const void* K, const void* V,
+                                                          const carnator_shape* s, void* O, float* LSE,
+                                                          void* ws, size_t ws_bytes, void* stream_) {
+    carnator_status st = check_shape(s, true);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !V || !O || !LSE) return CARNATOR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(LSE, 4)) return CARNATOR_ERR_INVALID_ARG;
+    AttnWs w;
+    st = attn_ws_check(s, ws, ws_bytes, &w);
+    if (st != CARNATOR_OK) return st;
+    const bool tc_ok = tcgen05_supported(s);
+    if (s->attn_impl == CARNATOR_IMPL_TCGEN05 && !tc_ok) return CARNATOR_ERR_UNSUPPORTED;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+
+    AttnArgs a;
+    a.Q = static_cast<const __nv_bfloat16*>(Q);
+    a.K = static_cast<const __nv_bfloat16*>(K);
+    a.V = static_cast<const __nv_bfloat16*>(V);
+    a.O = static_cast<__nv_bfloat16*>(O);
+    a.LSE = LSE;
+    for (int i = 0; i < 3; ++i) { a.qs[i] = s->q_stride[i]; a.ks[i] = s->k_stride[i]; a.vs[i] = s->v_stride[i]; a.os[i] = s->o_stride[i]; }
+    a.counts = w.counts; a.order = w.order; a.lists = w.lists; a.hdr = w.hdr;
+    a.B = s->B; a.H = s->H; a.N = s->N;
+    a.nqb = ceil_div(s->N, s->block_q); a.nkb = ceil_div(s->N, s->block_k);
+    a.block_q = s->block_q; a.block_k = s->block_k;
+    a.scale_log2 = effective_scale(s) * kLog2e;
+
+    const bool use_tc = tc_ok && s->attn_impl != CARNATOR_IMPL_PORTABLE;
+    if (use_tc) {
+        long long n = 0;
+        st = launch_tcgen05(a, s, stream, g_cuda_error, sizeof(g_cuda_error), &n);
+        g_launches.fetch_add(n, std::memory_order_relaxed);
+        return st;
+    }
+    if (s->D == 128 && s->block_q == 128) return launch_portable<128, 128>(a, stream);
+    if (s->D == 128 && s->block_q == 64) return launch_portable<128, 64>(a, stream);
+    if (s->D == 64 && s->block_q == 128) return launch_portable<64, 128>(a, stream);
+    return launch_portable<64, 64>(a, stream);
+}
+
+extern "C" carnator_status carnator_sparse_attn(const void* Q, const void* K, const void* V, const uint8_t* mask,
+                                                const uint8_t* recompute_rows, const carnator_shape* s, void* O,
+                                                float* LSE, void* ws, size_t ws_bytes, void* stream) {
+    // validate everything before the first launch
+    carnator_status st = check_shape(s, true);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !V || !O || !LSE || !mask) return CARNATOR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(LSE, 4)) return CARNATOR_ERR_INVALID_ARG;
+    if (s->attn_impl == CARNATOR_IMPL_TCGEN05 && !tcgen05_supported(s)) return CARNATOR_ERR_UNSUPPORTED;
+    st = carnator_compact_mask(mask, recompute_rows, s, ws, ws_bytes, stream);
+    if (st != CARNATOR_OK) return st;
+    return carnator_sparse_attn_compacted(Q, K, V, s, O, LSE, ws, ws_bytes, stream);
+}
+
+extern "C" carnator_status carnator_compacted_tiles(const carnator_shape* s, const void* ws, size_t ws_bytes,
+                                                    void* stream_, int64_t* tiles) {
+    carnator_status st = check_shape(s, true);
+    if (st != CARNATOR_OK) return st;
+    if (!tiles) return CARNATOR_ERR_INVALID_ARG;
+    AttnWs w;
+    st = attn_ws_check(s, const_cast<void*>(ws), ws_bytes, &w);
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    WsHeader h;
+    CUDA_TRY(cudaMemcpyAsync(&h, w.hdr, sizeof(WsHeader), cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    *tiles = int64_t(h.tiles);
+    return CARNATOR_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// host-buffer forms
+// ------------------------------------------------------------------------------------------------
+namespace {
+struct HostArena {
+    char *Q, *K, *V, *O;
+    float* LSE;
+    uint8_t *mask, *rec;
+    void* ws;
+    size_t ws_bytes, bytes;
+};
+HostArena attn_arena_layout(void* base, const carnator_shape* s) {
+    HostArena a;
+    char* p = static_cast<char*>(base);
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    const size_t t = align256(size_t(s->B) * s->H * s->N * s->D * 2);
+    size_t off = 0;
+    a.Q = p + off; off += t;
+    a.K = p + off; off += t;
+    a.V = p + off; off += t;
+    a.O = p + off; off += t;
+    a.LSE = reinterpret_cast<float*>(p + off); off += align256(size_t(s->B) * s->H * s->N * 4);
+    a.mask = reinterpret_cast<uint8_t*>(p + off); off += align256(size_t(s->B) * s->H * nqb * nkb);
+    a.rec = reinterpret_cast<uint8_t*>(p + off); off += align256(size_t(s->B) * nqb);
+    a.ws = p + off;
+    a.ws_bytes = attn_ws_layout(nullptr, s->B, s->H, nqb, nkb).bytes;
+    off += a.ws_bytes;
+    a.bytes = off;
+    return a;
+}
+void contiguous_strides(carnator_shape* c) {
+    const int64_t n = c->N, d = c->D, h = c->H;
+    int64_t st[3] = {h * n * d, n * d, d};
+    for (int i = 0; i < 3; ++i) c->q_stride[i] = c->k_stride[i] = c->v_stride[i] = c->o_stride[i] = st[i];
+}
+}  // namespace
+
+extern "C" size_t carnator_attn_host_arena_bytes(const carnator_shape* s_in) {
+    if (!s_in) return 0;
+    carnator_shape s = *s_in;
+    contiguous_strides(&s);
+    if (check_shape(&s, true) != CARNATOR_OK) return 0;
+    return attn_arena_layout(nullptr, &s).bytes;
+}
+
+extern "C" carnator_status carnator_sparse_attn_host(const void* Q, const void* K, const void* V, const uint8_t* mask,
+                                                     const uint8_t* recompute_rows, const carnator_shape* s_in,
+                                                     void* O, float* LSE, void* arena, size_t arena_bytes,
+                                                     void* stream_) {
+    if (!s_in) return CARNATOR_ERR_INVALID_ARG;
+    carnator_shape s = *s_in;
+    contiguous_strides(&s);
+    carnator_status st = check_shape(&s, true);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !V || !mask || !O || !LSE) return CARNATOR_ERR_INVALID_ARG;
+    if (!arena || !aligned(arena, 256)) return CARNATOR_ERR_WORKSPACE;
+    HostArena a = attn_arena_layout(arena, &s);
+    if (arena_bytes < a.bytes) return CARNATOR_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int nqb = ceil_div(s.N, s.block_q), nkb = ceil_div(s.N, s.block_k);
+    const size_t t = size_t(s.B) * s.H * s.N * s.D * 2;
+    CUDA_TRY(cudaMemcpyAsync(a.Q, Q, t, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(a.K, K, t, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(a.V, V, t, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(a.mask, mask, size_t(s.B) * s.H * nqb * nkb, cudaMemcpyHostToDevice, stream));
+    if (recompute_rows) CUDA_TRY(cudaMemcpyAsync(a.rec, recompute_rows, size_t(s.B) * nqb, cudaMemcpyHostToDevice, stream));
+    st = carnator_sparse_attn(a.Q, a.K, a.V, a.mask, recompute_rows ? a.rec : nullptr, &s, a.O, a.LSE, a.ws, a.ws_bytes, stream_);
+    if (st != CARNATOR_OK) return st;
+    CUDA_TRY(cudaMemcpyAsync(O, a.O, t, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaMemcpyAsync(LSE, a.LSE, size_t(s.B) * s.H * s.N * 4, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return carnator_query_status(a.ws, stream_);
+}
+
+extern "C" size_t carnator_build_host_arena_bytes(const carnator_shape* s_in, const carnator_build_params* p) {
+    if (!s_in) return 0;
+    carnator_shape s = *s_in;
+    contiguous_strides(&s);
+    if (check_shape(&s, false) != CARNATOR_OK || check_params(p) != CARNATOR_OK) return 0;
+    const int nqb = ceil_div(s.N, s.block_q), nkb = ceil_div(s.N, s.block_k);
+    const size_t t = align256(size_t(s.B) * s.H * s.N * s.D * 2);
+    return 2 * t + align256(size_t(s.B) * s.H * nqb * nkb) + build_ws_layout(nullptr, s.B, s.H, nqb, nkb, s.D).bytes;
+}
+
+extern "C" carnator_status carnator_build_connectivity_host(const void* Q, const void* K, const carnator_shape* s_in,
+                                                            const carnator_build_params* p, uint8_t* mask,
+                                                            void* arena, size_t arena_bytes, void* stream_) {
+    if (!s_in) return CARNATOR_ERR_INVALID_ARG;
+    carnator_shape s = *s_in;
+    contiguous_strides(&s);
+    carnator_status st = check_shape(&s, false);
+    if (st != CARNATOR_OK) return st;
+    st = check_params(p);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !mask) return CARNATOR_ERR_INVALID_ARG;
+    if (!arena || !aligned(arena, 256)) return CARNATOR_ERR_WORKSPACE;
+    const size_t need = carnator_build_host_arena_bytes(&s, p);
+    if (arena_bytes < need) return CARNATOR_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int nqb = ceil_div(s.N, s.block_q), nkb = ceil_div(s.N, s.block_k);
+    const size_t t = size_t(s.B) * s.H * s.N * s.D * 2, ta = align256(t);
+    const size_t mbytes = size_t(s.B) * s.H * nqb * nkb;
+    char* base = static_cast<char*>(arena);
+    char* dQ = base;
+    char* dK = base + ta;
+    uint8_t* dM = reinterpret_cast<uint8_t*>(base + 2 * ta);
+    void* ws = base + 2 * ta + align256(mbytes);
+    const size_t ws_bytes = need - (2 * ta + align256(mbytes));
+    CUDA_TRY(cudaMemcpyAsync(dQ, Q, t, cudaMemcpyHostToDevice, stream));
+    CUDA_TRY(cudaMemcpyAsync(dK, K, t, cudaMemcpyHostToDevice, stream));
+    st = carnator_build_connectivity(dQ, dK, &s, p, dM, nullptr, ws, ws_bytes, stream_);
+    if (st != CARNATOR_OK) return st;
+    CUDA_TRY(cudaMemcpyAsync(mask, dM, mbytes, cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    return carnator_query_status(ws, stream_);
+}
+
+// ------------------------------------------------------------------------------------------------
+// status
+// ------------------------------------------------------------------------------------------------
+extern "C" carnator_status carnator_query_status(void* ws, void* stream_) {
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    WsHeader h;
+    CUDA_TRY(cudaMemcpyAsync(&h, ws, sizeof(WsHeader), cudaMemcpyDeviceToHost, stream));
+    CUDA_TRY(cudaStreamSynchronize(stream));
+    if (h.status != 0) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "device status %d info %d %d %d", h.status, h.info[0], h.info[1], h.info[2]);
+        CUDA_TRY(cudaMemsetAsync(ws, 0, 16, stream));
+        CUDA_TRY(cudaStreamSynchronize(stream));
+        if (h.status == CARNATOR_ERR_DEVICE_TIMEOUT || h.status == CARNATOR_ERR_DEVICE_CHECK) return carnator_status(h.status);
+        return CARNATOR_ERR_DEVICE_CHECK;
+    }
+    return CARNATOR_OK;
+}
+
+extern "C" const char* carnator_status_string(carnator_status s) {
+    switch (s) {
+        case CARNATOR_OK: return "ok";
+        case CARNATOR_ERR_INVALID_ARG: return "invalid argument";
+        case CARNATOR_ERR_UNSUPPORTED: return "unsupported shape or device";
+        case CARNATOR_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case CARNATOR_ERR_CUDA: return "CUDA call failed";
+        case CARNATOR_ERR_DEVICE_TIMEOUT: return "bounded device-side wait expired";
+        case CARNATOR_ERR_DEVICE_CHECK: return "device-side consistency check failed";
+    }
+    return "unknown status";
+}
+
+extern "C" const char* carnator_last_cuda_error(void) { return g_cuda_error; }
+extern "C" int64_t carnator_kernel_launches(void) { return g_launches.load(std::memory_order_relaxed); }
+extern "C" int32_t carnator_version(void) { return 1; }

@@ -1,0 +1,171 @@
+"""GPU parity of carnator_sparse_attn against the CPU oracle, through the C ABI.
+
+Small cases are compared element by element; the full-size workloads are run in the launch
+configuration the benchmark times and compared on sampled (head, query block) rows, each of
+which the oracle computes independently.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import carnator_oracle as orc
+from paper_2609_32420_b200 import carnator as cn
+from paper_2609_32420_b200 import workloads as wl
+from tests.gpu_util import gather_rows, o_to_host, pick_rows, to_dev
+from tests.helpers import check_attention, rand_bits
+
+pytestmark = pytest.mark.gpu
+
+IMPLS = [cn.IMPL_PORTABLE, cn.IMPL_TCGEN05]
+IMPL_IDS = ["portable", "tcgen05"]
+
+
+def _tc_ok(block_q, block_k):
+    return block_q == 128 and block_k == 128
+
+
+def _run(Qb, Kb, Vb, N, n_text, T, Hg, Wg, bq, bk, mask, rec, impl, scale=0.0):
+    B, H, _, D = Qb.shape
+    Q, K, V = to_dev(Qb), to_dev(Kb), to_dev(Vb)
+    shape = cn.make_shape(B, H, N, D, n_text, T, Hg, Wg, bq, bk, Q, K, V, None, softmax_scale=scale, attn_impl=impl)
+    m = torch.from_numpy(mask).cuda()
+    r = torch.from_numpy(rec).cuda() if rec is not None else None
+    O, L, ws = cn.sparse_attn(Q, K, V, m, r, shape)
+    assert cn.query_status(ws) == cn.OK, cn.last_cuda_error()
+    return O, L, ws, shape
+
+
+@pytest.mark.parametrize("impl", IMPLS, ids=IMPL_IDS)
+def test_tiny_workload_full_compare(impl):
+    w = wl.get("tiny")
+    Qb, Kb, Vb = wl.gen_qkv(w)
+    bp = w.build
+    mask, _, _, _ = orc.build_connectivity(Qb, Kb, w.N, w.n_text, w.T, w.Hg, w.Wg, w.block, w.block, w.scale,
+                                           bp.mode, bp.keep_ratio, bp.mass, bp.window_frames, bp.text_dense,
+                                           bp.count_includes_forced)
+    rec = wl.gen_recompute_rows(w)
+    assert rec.sum() == 3
+    if impl == cn.IMPL_TCGEN05:
+        with pytest.raises(cn.CarnatorError) as e:
+            _run(Qb, Kb, Vb, w.N, 0, w.T, w.Hg, w.Wg, 64, 64, mask, rec, impl)
+        assert e.value.status == cn.ERR_UNSUPPORTED      # 64-token blocks run on the portable kernel
+        return
+    O, L, _, _ = _run(Qb, Kb, Vb, w.N, 0, w.T, w.Hg, w.Wg, 64, 64, mask, rec, impl)
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, w.N, 64, 64, w.scale, mask, rec)
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "tiny")
+
+
+CASES = [
+    # name, base workload, shrink kwargs, mask density
+    ("wan_ragged", "wan1p3b_480p", dict(H=2, T=3), 0.3),          # N=4680: 36 full blocks + 72-token tail, padded buffer
+    ("cog_text_d64", "cogvideox5b", dict(H=3, T=2), 0.4),         # N=2926, D=64, text prefix straddles block 1
+    ("hunyuan_tail16", "hunyuan_720p", dict(H=2, T=1), 0.25),     # N=3856: tail of 16 tokens
+]
+
+
+@pytest.mark.parametrize("impl", IMPLS, ids=IMPL_IDS)
+@pytest.mark.parametrize("name,base,kw,density", CASES, ids=[c[0] for c in CASES])
+def test_midsize_random_masks_full_compare(name, base, kw, density, impl):
+    w = wl.shrunk(wl.get(base), **kw)
+    Qb, Kb, Vb = wl.gen_qkv(w)
+    mask = wl.gen_random_mask(w, density, seed=1)
+    mask[0, 0, 2, :] = 0                                   # an empty row
+    mask[0, 1, 3, :] = 0
+    mask[0, 1, 3, w.nkb - 1] = 1                           # a row that sees only the ragged tail block
+    rec = wl.gen_recompute_rows(w)
+    rec[0, 2] = 0
+    rec[0, 3] = 0
+    O, L, ws, shape = _run(Qb, Kb, Vb, w.N, w.n_text, w.T, w.Hg, w.Wg, w.block, w.block, mask, rec, impl)
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, w.N, w.block, w.block, w.scale, mask, rec)
+    assert np.isneginf(L_ref[0, 0, 2 * w.block]).all()
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, name)
+    eff = (mask != 0) | (rec != 0)[:, None, :, None]
+    assert cn.compacted_tiles(shape, ws) == int(eff.sum())
+
+
+@pytest.mark.parametrize("impl", IMPLS, ids=IMPL_IDS)
+@pytest.mark.parametrize("D,bq,bk,N", [(64, 64, 128, 1000), (128, 128, 64, 777), (128, 64, 64, 130),
+                                       (64, 128, 128, 100), (128, 128, 128, 1), (128, 128, 128, 1153)])
+def test_block_and_head_dim_combinations(D, bq, bk, N, impl):
+    if impl == cn.IMPL_TCGEN05 and not _tc_ok(bq, bk):
+        pytest.skip("tcgen05 kernel takes 128-token blocks")
+    rng = np.random.default_rng(N + D)
+    B, H = 2, 2
+    Qb, Kb, Vb = (rand_bits(rng, (B, H, N, D)) for _ in range(3))
+    nqb, nkb = -(-N // bq), -(-N // bk)
+    mask = (rng.random((B, H, nqb, nkb)) < 0.5).astype(np.uint8)
+    rec = (rng.random((B, nqb)) < 0.2).astype(np.uint8)
+    O, L, _, _ = _run(Qb, Kb, Vb, N, 0, 1, 1, N, bq, bk, mask, rec, impl, scale=0.11)
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, N, bq, bk, 0.11, mask, rec)
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, f"D{D} bq{bq} bk{bk} N{N}")
+
+
+@pytest.mark.parametrize("impl", IMPLS, ids=IMPL_IDS)
+def test_degenerate_masks_and_large_scores(impl):
+    rng = np.random.default_rng(5)
+    N, D = 900, 128
+    Qb, Kb, Vb = (rand_bits(rng, (1, 2, N, D), scale=s) for s in (4.0, 4.0, 1.0))   # scores up to ~ +-60
+    nb = -(-N // 128)
+    zero = np.zeros((1, 2, nb, nb), dtype=np.uint8)
+    O, L, _, _ = _run(Qb, Kb, Vb, N, 0, 1, 1, N, 128, 128, zero, None, impl)
+    assert (O.float() == 0).all() and torch.isneginf(L).all()           # nothing to attend to
+    ones = np.ones_like(zero)
+    O, L, _, _ = _run(Qb, Kb, Vb, N, 0, 1, 1, N, 128, 128, ones, None, impl)
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, N, 128, 128, 1.0 / np.sqrt(D), ones, None)
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "dense, large scores")
+    # recompute rows make the mask contents irrelevant
+    rec = np.ones((1, nb), dtype=np.uint8)
+    O2, L2, _, _ = _run(Qb, Kb, Vb, N, 0, 1, 1, N, 128, 128, zero, rec, impl)
+    assert torch.equal(O, O2) and torch.equal(L, L2)
+
+
+@pytest.mark.parametrize("impl", IMPLS, ids=IMPL_IDS)
+def test_strided_inputs_and_rows_past_n_untouched(impl):
+    """Q/K/V as slices of one packed [B, rows, 3, H, D] buffer (token-major strides); O rows >= N keep their content."""
+    rng = np.random.default_rng(6)
+    B, H, N, D, rows = 1, 3, 500, 128, 512
+    packed = rand_bits(rng, (B, rows, 3, H, D))
+    P = to_dev(packed)
+    Q, K, V = (P[:, :, i].permute(0, 2, 1, 3) for i in range(3))        # [B,H,rows,D] views
+    O = torch.full((B, H, rows, D), 7.0, dtype=torch.bfloat16, device="cuda")
+    shape = cn.make_shape(B, H, N, D, 0, 1, 1, N, 128, 128, Q, K, V, O, attn_impl=impl)
+    nb = 4
+    mask = (rng.random((B, H, nb, nb)) < 0.6).astype(np.uint8)
+    O, L, ws = cn.sparse_attn(Q, K, V, torch.from_numpy(mask).cuda(), None, shape, O=O)
+    assert cn.query_status(ws) == cn.OK
+    assert (O[:, :, N:].float() == 7.0).all()
+    Qb, Kb, Vb = (np.ascontiguousarray(packed[:, :, i].transpose(0, 2, 1, 3)) for i in range(3))
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, N, 128, 128, 1.0 / np.sqrt(D), mask, None)
+    check_attention(o_to_host(O[:, :, :N]), L.cpu().numpy(), O_ref, L_ref, "strided")
+
+
+FULL = [("wan1p3b_480p", None), ("cogvideox5b", None), ("wan14b_720p", None), ("hunyuan_720p", 0.10)]
+
+
+@pytest.mark.parametrize("name,density", FULL, ids=[f[0] for f in FULL])
+def test_full_size_workload_sampled_rows(name, density):
+    """Whole layer at the benchmark's launch configuration (mask from the GPU builder on the
+    historical Q/K pair); sampled (head, query block) rows against the oracle."""
+    w = wl.get(name)
+    if density is not None:
+        w = w.replace(build=dataclasses.replace(w.build, keep_ratio=density))
+    heads = [(0, 0), (0, w.H - 1)]
+    Q, K, V = (to_dev(wl.gen_tensor(w, t)) for t in "QKV")
+    Qh, Kh = (to_dev(wl.gen_tensor(w, t, "history")) for t in "QK")
+    shape = cn.shape_of(w, Q, K, V, None, attn_impl=cn.IMPL_AUTO)
+    mask_dev, _ = cn.build_connectivity(Qh, Kh, cn.shape_of(w, Qh, Kh), cn.params_of(w.build))
+    del Qh, Kh
+    rec = wl.gen_recompute_rows(w)
+    O, L, ws = cn.sparse_attn(Q, K, V, mask_dev, torch.from_numpy(rec).cuda(), shape)
+    assert cn.query_status(ws) == cn.OK, cn.last_cuda_error()
+    mask = mask_dev.cpu().numpy()
+    rows = pick_rows(mask, rec, w, heads, extra_per_head=1, seed=w.cfg)
+    # the oracle needs only the sampled heads on the host
+    Qb, Kb, Vb = wl.gen_qkv(w, heads=heads)
+    O_ref, L_ref = orc.attention_rows(Qb, Kb, Vb, w.N, w.block, w.block, w.scale, mask, rec, rows)
+    O_g, L_g = gather_rows(O, L, rows, w)
+    check_attention(O_g, L_g, O_ref, L_ref, name)
+    # properties that hold at any size: every valid row finite, no row past N touched is checked above by shape
+    assert torch.isfinite(O.float()).all() and torch.isfinite(L).all()

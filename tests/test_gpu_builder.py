@@ -1,0 +1,112 @@
+"""GPU parity of carnator_build_connectivity against the builder oracle, through the C ABI.
+
+Bar: the block mask is bit-exact except for blocks whose fp32 pooled score (the oracle's) lies
+within 1e-4 of the row's selection threshold; always-kept blocks must match; in top-k mode the
+per-row count must match.  Pooled scores themselves are compared to 2e-5 absolute.
+"""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import carnator_oracle as orc
+from paper_2609_32420_b200 import carnator as cn
+from paper_2609_32420_b200 import workloads as wl
+from tests.gpu_util import to_dev
+from tests.helpers import check_mask
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle(w, Qb, Kb, heads=None):
+    bp = w.build
+    return orc.build_connectivity(Qb, Kb, w.N, w.n_text, w.T, w.Hg, w.Wg, w.block, w.block, w.scale,
+                                  bp.mode, bp.keep_ratio, bp.mass, bp.window_frames, bp.text_dense,
+                                  bp.count_includes_forced, heads=heads)
+
+
+def _gpu(w, Qb, Kb):
+    Q, K = to_dev(Qb), to_dev(Kb)
+    shape = cn.shape_of(w, Q, K)
+    scores = torch.empty((w.B, w.H, w.nqb, w.nkb), dtype=torch.float32, device="cuda")
+    mask, ws = cn.build_connectivity(Q, K, shape, cn.params_of(w.build), pooled_scores=scores)
+    assert cn.query_status(ws) == cn.OK
+    return mask.cpu().numpy(), scores.cpu().numpy()
+
+
+def _compare(w, Qb, Kb, heads=None, what=""):
+    mask_g, scores_g = _gpu(w, Qb, Kb)
+    mask_r, scores_r, theta, F = _oracle(w, Qb, Kb, heads)
+    if heads is not None:
+        sel = np.zeros((w.B, w.H), dtype=bool)
+        for (b, h) in heads:
+            sel[b, h] = True
+        mask_g = np.where(sel[:, :, None, None], mask_g, 0)
+        scores_g = np.where(sel[:, :, None, None], scores_g, 0)
+    assert np.abs(scores_g - scores_r).max() <= 2e-5, f"{what}: pooled scores differ by {np.abs(scores_g - scores_r).max()}"
+    return check_mask(mask_g, mask_r, scores_r, theta, F, topk_mode=(w.build.mode == wl.MODE_TOPK), what=what)
+
+
+def test_tiny_topk():
+    w = wl.get("tiny")
+    Qb, Kb, _ = wl.gen_qkv(w)
+    _compare(w, Qb, Kb, what="tiny")
+
+
+@pytest.mark.parametrize("name,kw", [
+    ("wan1p3b_480p", dict(H=2, T=3)),
+    ("cogvideox5b", dict(H=3, T=2)),
+    ("hunyuan_720p", dict(H=2, T=1)),
+])
+def test_midsize_window_text_rules(name, kw):
+    w = wl.shrunk(wl.get(name), **kw)
+    Qb, Kb, _ = wl.gen_qkv(w, "history")
+    _compare(w, Qb, Kb, what=name)
+
+
+@pytest.mark.parametrize("mass", [0.5, 0.9, 0.95])
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("wan1p3b_480p", dict(H=2, T=4))])
+def test_cumulative_mass_mode(name, kw, mass):
+    w = wl.get(name)
+    if kw:
+        w = wl.shrunk(w, **kw)
+    w = w.replace(build=dataclasses.replace(w.build, mode=wl.MODE_CUMMASS, mass=mass))
+    Qb, Kb, _ = wl.gen_qkv(w, "history")
+    _compare(w, Qb, Kb, what=f"{name} cummass {mass}")
+
+
+def test_ties_are_broken_by_lower_block_index():
+    """Identical key blocks give identical pooled scores: the lower index must win, exactly as the oracle does."""
+    w = wl.shrunk(wl.get("wan1p3b_480p"), H=1, T=2).replace(
+        build=wl.BuildParams(keep_ratio=0.3, window_frames=-1))
+    Qb, Kb, _ = wl.gen_qkv(w, "history")
+    blk = Kb[:, :, :128].copy()
+    for J in range(w.N // 128):
+        Kb[:, :, J * 128:(J + 1) * 128] = blk
+    mask_g, _ = _gpu(w, Qb, Kb)
+    mask_r, _, _, _ = _oracle(w, Qb, Kb)
+    full = w.N // 128
+    np.testing.assert_array_equal(mask_g[..., :full], mask_r[..., :full])
+
+
+def test_keep_ratio_one_is_all_ones():
+    w = wl.shrunk(wl.get("hunyuan_720p"), H=1, T=1).replace()
+    w = w.replace(build=dataclasses.replace(w.build, keep_ratio=1.0))
+    Qb, Kb, _ = wl.gen_qkv(w, "history")
+    mask_g, _ = _gpu(w, Qb, Kb)
+    assert (mask_g == 1).all()
+
+
+FULL = ["wan1p3b_480p", "cogvideox5b", "wan14b_720p", "hunyuan_720p"]
+
+
+@pytest.mark.parametrize("name", FULL)
+def test_full_size_masks_on_sampled_heads(name):
+    """Full-size launch; the oracle checks two heads in full (every row, every block)."""
+    w = wl.get(name)
+    heads = [(0, 1), (0, w.H - 2)]
+    Qb = wl.gen_tensor(w, "Q", "history")
+    Kb = wl.gen_tensor(w, "K", "history")
+    n_excused = _compare(w, Qb, Kb, heads=heads, what=name)
+    assert n_excused <= 8
