@@ -1,10 +1,489 @@
-// placeholder until the tcgen05 kernel lands
+// Block-sparse attention on the 5th-generation tensor cores: TMA loads of the listed K/V tiles,
+// tcgen05.mma with S = Q K^T and O += P V accumulated in tensor memory, online softmax in the
+// consumer warps.  One CTA per (batch, head, query block) of 128 queries; key blocks of 128.
+// Paper: Section 3.3, "Historical Sparse-Connectivity Reuse" (only the block pairs the historical
+// structure lists are evaluated; Q, K, V are the target's own).
+//
+// Warp roles (192 threads):
+//   warps 0-3  softmax + epilogue; warp w owns tensor-memory lanes 32w..32w+31 = query rows
+//   warp 4     TMA producer (one lane)
+//   warp 5     tensor-memory allocation, MMA issue (one lane)
+// Tensor memory (256 columns per CTA, two CTAs per SM): S fp32 at columns [0,128), P bf16 packed
+// into columns [0,64) once S has been read, O fp32 at columns [128,128+D).
+// Every wait on an mbarrier is bounded; on expiry the role records CARNATOR_ERR_DEVICE_TIMEOUT in
+// the workspace header, raises a CTA-wide abort flag, and every role drains and returns.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 #include "attn_portable.cuh"
+
 namespace carnator {
-inline bool tcgen05_supported(const carnator_shape*) { return false; }
-inline carnator_status launch_tcgen05(const AttnArgs&, const carnator_shape*, cudaStream_t, char*, size_t, long long*) {
-    return CARNATOR_ERR_UNSUPPORTED;
+namespace tc {
+
+constexpr int kBlock = 128;            // query rows per CTA = keys per tile
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 256;
+constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
+constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8, well inside bf16/fp32 range
+
+// ---- small PTX wrappers -----------------------------------------------------------------------
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up after ~2 s (or when another role has aborted) and raises the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 0; it < (1u << 30); ++it) {
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 255u) == 255u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > 2000000000ull) break;
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
+                                            int c0, int c1, int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void prefetch_tmap(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr),
+          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr),
+          "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
+// ---- descriptors --------------------------------------------------------------------------------
+// Shared-memory matrix descriptor, 128-byte swizzle: start address, leading / stride byte offsets
+// (all in 16-byte units), descriptor version 1 (bit 46), layout type 2 = SWIZZLE_128B (bits 61-63).
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return uint64_t((addr & 0x3FFFFu) >> 4)
+         | (uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16)
+         | (uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32)
+         | (1ull << 46)
+         | (2ull << 61);
+}
+// Instruction descriptor for kind::f16: fp32 accumulator, bf16 x bf16, M x N, B operand major-ness.
+__host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
+}
+
+template <int D, int STAGES>
+struct Cfg {
+    static constexpr int kBoxes = D / 64;                       // 64-element (128-byte) boxes per row
+    static constexpr uint32_t kBoxBytes = kBlock * 128;         // 128 rows x 128 B
+    static constexpr uint32_t kTileBytes = kBoxes * kBoxBytes;  // one 128 x D bf16 tile
+    static constexpr uint32_t kOffQ = 0;
+    static constexpr uint32_t kOffK = kTileBytes;
+    static constexpr uint32_t kOffV = kOffK + STAGES * kTileBytes;
+    static constexpr uint32_t kOffBar = kOffV + STAGES * kTileBytes;
+    static constexpr uint32_t kNeeded = kOffBar + 256 + 1024;   // barriers + slack to align the base to 1 KiB
+    // request enough that at most two CTAs fit an SM (two x 256 tensor-memory columns)
+    static constexpr uint32_t kSmemBytes = kNeeded > 78 * 1024 ? kNeeded : 78 * 1024;
+};
+
+struct TcParams {
+    AttnArgs a;
+};
+
+template <int D, int STAGES>
+__global__ void __launch_bounds__(kThreads, 2)
+attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
+                    const __grid_constant__ CUtensorMap mapV, const AttnArgs a) {
+    using C = Cfg<D, STAGES>;
+    extern __shared__ unsigned char smem_dyn[];
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int b = blockIdx.z, h = blockIdx.y;
+    const int64_t bh = int64_t(b) * a.H + h;
+    const int I = a.order[bh * a.nqb + blockIdx.x];
+    const int count = a.counts[bh * a.nqb + I];
+    const int32_t* list = a.lists + (bh * a.nqb + I) * int64_t(a.nkb);
+    const int q0 = I * kBlock;
+
+    if (count == 0) {                       // nothing to attend to: O = 0, LSE = -inf
+        if (tid < kBlock && q0 + tid < a.N) {
+            __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(q0 + tid) * a.os[2];
+#pragma unroll
+            for (int c = 0; c < D / 8; ++c) *reinterpret_cast<uint4*>(op + c * 8) = make_uint4(0, 0, 0, 0);
+            a.LSE[bh * a.N + q0 + tid] = -INFINITY;
+        }
+        return;
+    }
+
+    const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
+    const uint32_t sQ = smem_base + C::kOffQ;
+    const uint32_t sK = smem_base + C::kOffK;
+    const uint32_t sV = smem_base + C::kOffV;
+    const uint32_t bars = smem_base + C::kOffBar;
+    // barrier slots (8 bytes each)
+    const uint32_t bar_q = bars;
+    const uint32_t bar_s = bars + 8;
+    const uint32_t bar_p = bars + 16;
+    const uint32_t bar_o = bars + 24;
+    const uint32_t bar_drain = bars + 32;
+    auto bar_kfull = [&](int s) { return bars + 64 + 8 * s; };
+    auto bar_kempty = [&](int s) { return bars + 64 + 8 * (STAGES + s); };
+    auto bar_vfull = [&](int s) { return bars + 64 + 8 * (2 * STAGES + s); };
+    auto bar_vempty = [&](int s) { return bars + 64 + 8 * (3 * STAGES + s); };
+    volatile int* abortp = &abort_flag;
+
+    if (tid == 0) {
+        abort_flag = 0;
+        mbar_init(bar_q, 1); mbar_init(bar_s, 1); mbar_init(bar_p, kBlock); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
+            mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 4 && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapV); }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    if (warp == 4) {
+        // ================= TMA producer =================
+        if (lane == 0) {
+            mbar_expect_tx(bar_q, C::kTileBytes);
+#pragma unroll
+            for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
+            bool ok = true;
+            int armed_k = -1, armed_v = -1;     // last tile whose loads were issued
+            for (int j = 0; j < count && ok; ++j) {
+                const int s = j % STAGES;
+                const uint32_t par = uint32_t(j / STAGES) & 1u;
+                const int J = list[j];
+                ok = mbar_wait(bar_kempty(s), par ^ 1u, abortp);
+                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, j, blockIdx.x); break; }
+                mbar_expect_tx(bar_kfull(s), C::kTileBytes);
+#pragma unroll
+                for (int x = 0; x < C::kBoxes; ++x)
+                    tma_load_4d(sK + s * C::kTileBytes + x * C::kBoxBytes, &mapK, bar_kfull(s), x * 64, J * kBlock, h, b);
+                armed_k = j;
+                ok = mbar_wait(bar_vempty(s), par ^ 1u, abortp);
+                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, j, blockIdx.x); break; }
+                mbar_expect_tx(bar_vfull(s), C::kTileBytes);
+#pragma unroll
+                for (int x = 0; x < C::kBoxes; ++x)
+                    tma_load_4d(sV + s * C::kTileBytes + x * C::kBoxBytes, &mapV, bar_vfull(s), x * 64, J * kBlock, h, b);
+                armed_v = j;
+            }
+            if (*abortp) {
+                // drain: copies in flight must land before the CTA gives its shared memory back
+                mbar_wait(bar_q, 0, abortp);
+                if (armed_k >= 0) mbar_wait(bar_kfull(armed_k % STAGES), uint32_t(armed_k / STAGES) & 1u, abortp);
+                if (armed_v >= 0) mbar_wait(bar_vfull(armed_v % STAGES), uint32_t(armed_v / STAGES) & 1u, abortp);
+            }
+        }
+    } else if (warp == 5) {
+        // ================= MMA issuer =================
+        if (lane == 0) {
+            constexpr uint32_t idesc_qk = instr_desc(kBlock, kBlock, 0);
+            constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
+            bool ok = mbar_wait(bar_q, 0, abortp);
+            if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
+            for (int j = 0; j < count && ok; ++j) {
+                const int s = j % STAGES;
+                const uint32_t par = uint32_t(j / STAGES) & 1u;
+                ok = mbar_wait(bar_kfull(s), par, abortp);
+                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, j, blockIdx.x); break; }
+                tc_fence_after();
+                // S = Q K^T : K-major operands, 16 elements of the head dimension per instruction
+#pragma unroll
+                for (int kk = 0; kk < D / 16; ++kk) {
+                    const uint32_t off = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
+                    mma_ss(tmem + kColS, smem_desc(sQ + off, 16, 1024), smem_desc(sK + s * C::kTileBytes + off, 16, 1024),
+                           idesc_qk, kk > 0);
+                }
+                tc_commit(bar_s);
+                tc_commit(bar_kempty(s));
+                ok = mbar_wait(bar_p, uint32_t(j) & 1u, abortp);
+                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, j, blockIdx.x); break; }
+                ok = mbar_wait(bar_vfull(s), par, abortp);
+                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 6, j, blockIdx.x); break; }
+                tc_fence_after();
+                // O += P V : P from tensor memory (16 keys = 8 packed columns per instruction),
+                // V tile as the MN-major B operand (rows = keys, 64-element chunks of the head dimension)
+#pragma unroll
+                for (int kk = 0; kk < kBlock / 16; ++kk) {
+                    mma_ts(tmem + kColO, tmem + kColP + kk * 8,
+                           smem_desc(sV + s * C::kTileBytes + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (j > 0) || (kk > 0));
+                }
+                tc_commit(bar_vempty(s));
+                if (j == count - 1) tc_commit(bar_o);
+            }
+            if (*abortp) {
+                // make sure no MMA is still running before tensor memory is released
+                tc_commit(bar_drain);
+                mbar_wait(bar_drain, 0, abortp);
+            }
+        }
+    } else {
+        // ================= softmax + epilogue (warps 0-3) =================
+        const uint32_t lane_base = uint32_t(warp * 32) << 16;
+        const int row = q0 + tid;
+        float m_used = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int j = 0; j < count; ++j) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_s, uint32_t(j) & 1u, abortp));   // warp-uniform: the loads below are collective
+            if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, j, blockIdx.x); break; }
+            tc_fence_after();
+            const int J = list[j];
+            const int nvalid = min(kBlock, a.N - J * kBlock);
+            float s[4][32];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tmem + lane_base + kColS + c * 32, s[c]);
+            tmem_wait_ld();
+            float mx = -INFINITY;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float v = s[c][i] * a.scale_log2;
+                    if (c * 32 + i >= nvalid) v = -INFINITY;
+                    s[c][i] = v;
+                    mx = fmaxf(mx, v);
+                }
+            }
+            // lazy rescale: the reference maximum only moves when it would grow by more than the threshold
+            const bool grow = (mx > m_used + kRescaleThreshold);     // first tile: m_used = -inf -> true
+            if (j == 0) {
+                m_used = mx;
+            } else if (__any_sync(0xffffffffu, grow)) {
+                // s_full(j) was committed after P V of tile j-1, so O is quiescent here
+                const float m_new = grow ? mx : m_used;
+                const float f = exp2f(m_used - m_new);
+#pragma unroll
+                for (int c = 0; c < D / 32; ++c) {
+                    float o[32];
+                    tmem_ld32(tmem + lane_base + kColO + c * 32, o);
+                    tmem_wait_ld();
+                    uint32_t r[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(o[i] * f);
+                    tmem_st32(tmem + lane_base + kColO + c * 32, r);
+                }
+                l_sum *= f;
+                m_used = m_new;
+            }
+            // P = exp2(s - m_used) as packed bf16 pairs into columns [0,64)
+            float part = 0.f;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float p0 = exp2f(s[c][2 * i] - m_used);
+                    const float p1 = exp2f(s[c][2 * i + 1] - m_used);
+                    part += p0 + p1;
+                    pk[i] = pack_bf16(p0, p1);
+                }
+                tmem_st16(tmem + lane_base + kColP + c * 16, pk);
+            }
+            l_sum += part;
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive(bar_p);
+        }
+        if (ok) {
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, 0, abortp));
+            if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 8, count, blockIdx.x);
+        }
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.f / l_sum;
+            __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(row) * a.os[2];
+#pragma unroll
+            for (int c = 0; c < D / 32; ++c) {
+                float o[32];
+                tmem_ld32(tmem + lane_base + kColO + c * 32, o);      // warp-collective: every lane takes part
+                tmem_wait_ld();
+                if (row < a.N) {
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        uint4 u;
+                        u.x = pack_bf16(o[8 * v + 0] * inv, o[8 * v + 1] * inv);
+                        u.y = pack_bf16(o[8 * v + 2] * inv, o[8 * v + 3] * inv);
+                        u.z = pack_bf16(o[8 * v + 4] * inv, o[8 * v + 5] * inv);
+                        u.w = pack_bf16(o[8 * v + 6] * inv, o[8 * v + 7] * inv);
+                        *reinterpret_cast<uint4*>(op + c * 32 + v * 8) = u;
+                    }
+                }
+            }
+            if (row < a.N) a.LSE[bh * a.N + row] = (m_used + log2f(l_sum)) * kLn2;
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// 4-D map over a [B,H,N,D] bf16 tensor with arbitrary (16-byte multiple) strides: box = 64 x 128 x 1 x 1,
+// 128-byte swizzle, rows >= N read as zero.
+inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, int D, const int64_t st[3]) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(N), cuuint64_t(H), cuuint64_t(B)};
+    // a stride of a size-1 axis is never used for addressing but must still be a valid value
+    const cuuint64_t row = cuuint64_t(st[2]) * 2;
+    cuuint64_t s_h = (H > 1 || st[1] > 0) ? cuuint64_t(st[1]) * 2 : row * N;
+    cuuint64_t s_b = (B > 1 || st[0] > 0) ? cuuint64_t(st[0]) * 2 : s_h * H;
+    if (s_h == 0) s_h = row * N;
+    if (s_b == 0) s_b = s_h * H;
+    cuuint64_t strides[3] = {row, s_h, s_b};
+    cuuint32_t box[4] = {64, cuuint32_t(kBlock), 1, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+}  // namespace tc
+
+inline bool tcgen05_supported(const carnator_shape* s) {
+    return s->block_q == tc::kBlock && s->block_k == tc::kBlock && (s->D == 64 || s->D == 128);
+}
+
+template <int D, int STAGES>
+inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+                                 cudaStream_t stream, char* err, size_t errlen) {
+    using C = tc::Cfg<D, STAGES>;
+    auto kern = tc::attn_tcgen05_kernel<D, STAGES>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmemBytes));
+    if (e != cudaSuccess) { snprintf(err, errlen, "cudaFuncSetAttribute(tcgen05): %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
+    dim3 grid(a.nqb, a.H, a.B);
+    kern<<<grid, tc::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, a);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { snprintf(err, errlen, "attn_tcgen05_kernel: %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
+    return CARNATOR_OK;
+}
+
+inline carnator_status launch_tcgen05(const AttnArgs& a, const carnator_shape* s, cudaStream_t stream,
+                                      char* err, size_t errlen, long long* launches) {
+    CUtensorMap mq, mk, mv;
+    if (!tc::make_map(&mq, a.Q, a.B, a.H, a.N, s->D, a.qs) || !tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks) ||
+        !tc::make_map(&mv, a.V, a.B, a.H, a.N, s->D, a.vs)) {
+        snprintf(err, errlen, "cuTensorMapEncodeTiled failed or is unavailable");
+        return CARNATOR_ERR_CUDA;
+    }
+    carnator_status st = (s->D == 128) ? launch_tc<128, 1>(a, mq, mk, mv, stream, err, errlen)
+                                       : launch_tc<64, 2>(a, mq, mk, mv, stream, err, errlen);
+    if (st == CARNATOR_OK) *launches = 1;
+    return st;
+}
+
+}  // namespace carnator
