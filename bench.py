@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--workload", default="wan14b_720p", choices=list(wl.WORKLOADS))
     ap.add_argument("--density", type=float, default=None, help="override the builder's keep ratio")
     ap.add_argument("--attn-impl", default="auto", choices=["auto", "portable", "tcgen05"])
+    ap.add_argument("--heads", type=int, default=None, help="run a slice with fewer heads (profiling captures)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -63,6 +64,8 @@ def workload_from_args(args) -> wl.Workload:
     w = wl.get(args.workload)
     if args.density is not None:
         w = w.replace(build=dataclasses.replace(w.build, keep_ratio=args.density))
+    if args.heads is not None:
+        w = w.replace(H=args.heads, name=f"{w.name}[H={args.heads}]")
     return w
 
 
