@@ -109,6 +109,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 #pragma unroll
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -322,25 +327,28 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tmem + lane_base + kColS + c * 32, s[c]);
             tmem_wait_ld();
-            float mx = -INFINITY;
+            if (nvalid < kBlock) {               // ragged last key block (warp-uniform): keys >= N never count
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float v = s[c][i] * a.scale_log2;
-                    if (c * 32 + i >= nvalid) v = -INFINITY;
-                    s[c][i] = v;
-                    mx = fmaxf(mx, v);
-                }
+                    for (int i = 0; i < 32; ++i)
+                        if (c * 32 + i >= nvalid) s[c][i] = -INFINITY;
             }
+            // row maximum of the raw scores (the scale is positive), four independent chains
+            float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+#pragma unroll
+                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], s[c][i]);
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
             // lazy rescale: the reference maximum only moves when it would grow by more than the threshold
-            const bool grow = (mx > m_used + kRescaleThreshold);     // first tile: m_used = -inf -> true
+            const bool grow = (mx > m_used + kRescaleThreshold);
             if (j == 0) {
                 m_used = mx;
             } else if (__any_sync(0xffffffffu, grow)) {
                 // s_full(j) was committed after P V of tile j-1, so O is quiescent here
                 const float m_new = grow ? mx : m_used;
-                const float f = exp2f(m_used - m_new);
+                const float f = ex2_approx(m_used - m_new);
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     float o[32];
@@ -354,21 +362,24 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 l_sum *= f;
                 m_used = m_new;
             }
-            // P = exp2(s - m_used) as packed bf16 pairs into columns [0,64)
-            float part = 0.f;
+            // P = exp2(s * scale - m_used): one FFMA + one MUFU per element, packed to bf16 pairs in columns [0,64)
+            const float neg_m = -m_used;
+            float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
-                    const float p0 = exp2f(s[c][2 * i] - m_used);
-                    const float p1 = exp2f(s[c][2 * i + 1] - m_used);
-                    part += p0 + p1;
+                    const float p0 = ex2_approx(fmaf(s[c][2 * i], a.scale_log2, neg_m));
+                    const float p1 = ex2_approx(fmaf(s[c][2 * i + 1], a.scale_log2, neg_m));
+                    part[i & 1] += p0;
+                    part[2 + (i & 1)] += p1;
                     pk[i] = pack_bf16(p0, p1);
                 }
                 tmem_st16(tmem + lane_base + kColP + c * 16, pk);
             }
-            l_sum += part;
+            const float part_sum = (part[0] + part[1]) + (part[2] + part[3]);
+            l_sum += part_sum;
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive(bar_p);
