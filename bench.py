@@ -208,6 +208,25 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# rank reduction (replicas only: the data path has no collective; only the timings are reduced)
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(values, device=None):
+    """Element-wise MAX over ranks of a list of floats (identity when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(v) for v in values]
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t.tolist()]
+
+
+def whole_job_tflops(flops_per_replica: float, world: int, ms_per_step: float) -> float:
+    """Every rank runs one replica of the workload; the job's throughput is all replicas' work over the slowest rank's time."""
+    return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
+
+
+# ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -303,12 +322,9 @@ def run_ours(args):
     ms_compact = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     ms_attn = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     ms_attn_min = float(np.min([e[2].elapsed_time(e[3]) for e in evs]))
-    if world > 1:
-        tt = torch.tensor([total_ms, ms_attn], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms, ms_attn = float(tt[0]), float(tt[1])
+    total_ms, ms_attn = max_over_ranks([total_ms, ms_attn], dev)
     ms_step = total_ms / args.steps
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = whole_job_tflops(flops, world, ms_step)
 
     # ---- end to end through the host-buffer calls --------------------------------------------------
     e2e = None
@@ -337,13 +353,10 @@ def run_ours(args):
         torch.cuda.synchronize()
         t1 = time.perf_counter()
         e2e_ms = 1e3 * (t1 - t0) / n_e2e
-        if world > 1:
-            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt[0])
+        e2e_ms = max_over_ranks([e2e_ms], dev)[0]
         tb = w.B * w.H * w.N * w.D * 2
         mb = w.B * w.H * w.nqb * w.nkb
-        e2e = {"value": world * flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+        e2e = {"value": whole_job_tflops(flops, world, e2e_ms), "unit": "TFLOP/s", "ms_per_step": e2e_ms,
                "steps": n_e2e, "h2d_bytes_per_step": 5 * tb + mb + w.B * w.nqb,
                "d2h_bytes_per_step": mb + tb + w.B * w.H * w.N * 4,
                "note": "carnator_build_connectivity_host + carnator_sparse_attn_host, pinned host buffers"}
