@@ -191,6 +191,42 @@ carnator_status carnator_build_connectivity_host(const void* Q, const void* K,
                                                  void* arena, size_t arena_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * carnator_sparse_attn_static -- carnator_sparse_attn for callers that cannot provide a workspace.
+ *
+ * (The paper has no counterpart for this call; it exists for deployment reasons only.)
+ *
+ * Some callers are not allowed to obtain device memory at the point where they call into this
+ * library: code running under a memory budget that was fixed at start-up, plugins whose host
+ * framework owns the allocator, and real-time loops in which cudaMalloc's implicit device
+ * synchronisation is not acceptable.  They still own their inputs and outputs, but have nowhere
+ * to put the compacted lists.  This form keeps that scratch in a fixed array that is part of the
+ * library image itself: CARNATOR_STATIC_SCRATCH_BYTES of device memory, reserved on every GPU
+ * the process uses the library on, from load until exit.
+ *
+ *   - Same arguments and results as carnator_sparse_attn, minus the workspace.
+ *   - The call allocates and frees nothing, on the device or through any library.
+ *   - A shape whose carnator_attn_workspace_bytes exceeds CARNATOR_STATIC_SCRATCH_BYTES is
+ *     rejected with CARNATOR_ERR_WORKSPACE before anything is launched;
+ *     carnator_last_cuda_error() then names both sizes.  (8 MiB covers e.g. B*H*nqb*nkb up to
+ *     about two million block pairs: the Wan-1.3B-shaped layer fits, the 14B-shaped one does not.)
+ *   - The first call on each device looks up the array's device address (once per device, with
+ *     that device current) and configures the kernels; make that first call outside of any
+ *     stream capture.
+ *   - All calls on one device share the one array.  It still holds the previous call's lists;
+ *     each call clears the header it relies on and rewrites every list entry it reads, so
+ *     back-to-back calls on one stream are safe.  Two calls that overlap on the GPU (different
+ *     streams, or different host threads without ordering) race on the array: order them.
+ *   - The device status word of this form lives inside the array and is not exposed; use the
+ *     workspace forms when bounded-wait diagnostics are needed.
+ * ------------------------------------------------------------------------ */
+#define CARNATOR_STATIC_SCRATCH_BYTES (8u << 20)
+
+carnator_status carnator_sparse_attn_static(const void* Q, const void* K, const void* V,
+                                            const uint8_t* mask, const uint8_t* recompute_rows,
+                                            const carnator_shape* shape,
+                                            void* O, float* LSE, void* stream);
+
+/* ------------------------------------------------------------------------
  * Status and diagnostics.
  * carnator_query_status synchronises `stream` and returns the status word that
  * kernels of earlier calls on this workspace may have set (CARNATOR_OK,

@@ -26,6 +26,7 @@ EXPORTS = [
     "carnator_sparse_attn", "carnator_compacted_tiles",
     "carnator_attn_host_arena_bytes", "carnator_sparse_attn_host",
     "carnator_build_host_arena_bytes", "carnator_build_connectivity_host",
+    "carnator_sparse_attn_static",
     "carnator_query_status", "carnator_status_string", "carnator_last_cuda_error",
     "carnator_kernel_launches", "carnator_version",
 ]
@@ -107,6 +108,8 @@ def lib() -> ctypes.CDLL:
     L.carnator_build_host_arena_bytes.argtypes = [ps, pp]
     L.carnator_build_connectivity_host.restype = ctypes.c_int
     L.carnator_build_connectivity_host.argtypes = [vp, vp, ps, pp, vp, vp, sz, vp]
+    L.carnator_sparse_attn_static.restype = ctypes.c_int
+    L.carnator_sparse_attn_static.argtypes = [vp, vp, vp, vp, vp, ps, vp, vp, vp]
     L.carnator_query_status.restype = ctypes.c_int
     L.carnator_query_status.argtypes = [vp, vp]
     L.carnator_status_string.restype = ctypes.c_char_p
@@ -284,3 +287,20 @@ def build_connectivity_host(Q, K, shape: Shape, params: BuildParams, mask, arena
     st = lib().carnator_build_connectivity_host(_ptr(Q), _ptr(K), ctypes.byref(shape), ctypes.byref(params),
                                                 _ptr(mask), _ptr(arena), arena.numel(), _stream(stream))
     _check(st, "carnator_build_connectivity_host")
+
+
+STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def sparse_attn_static(Q, K, V, mask, recompute_rows, shape: Shape, O, LSE, stream=None):
+    """carnator_sparse_attn_static: no workspace argument -- the library's built-in scratch array is used.
+
+    For callers that must not allocate device memory when they call (fixed memory budgets, hosts that own
+    the allocator, latency-critical loops).  O and LSE must be passed in; nothing is allocated here either.
+    Shapes whose workspace exceeds STATIC_SCRATCH_BYTES raise with CARNATOR_ERR_WORKSPACE.  Calls share the
+    one array per device: keep them ordered on the GPU.
+    """
+    shape.o_stride = (ctypes.c_int64 * 3)(*O.stride()[:3])
+    st = lib().carnator_sparse_attn_static(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), _ptr(recompute_rows),
+                                           ctypes.byref(shape), _ptr(O), _ptr(LSE), _stream(stream))
+    _check(st, "carnator_sparse_attn_static")

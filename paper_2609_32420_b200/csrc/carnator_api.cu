@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "carnator.h"
 #include "common.cuh"
@@ -423,6 +424,50 @@ extern "C" carnator_status carnator_build_connectivity_host(const void* Q, const
     CUDA_TRY(cudaMemcpyAsync(mask, dM, mbytes, cudaMemcpyDeviceToHost, stream));
     CUDA_TRY(cudaStreamSynchronize(stream));
     return carnator_query_status(ws, stream_);
+}
+
+// ------------------------------------------------------------------------------------------------
+// static-scratch form: for callers that may not obtain device memory (fixed budgets, plugins whose host
+// owns the allocator, loops that cannot tolerate cudaMalloc's synchronisation).  The scratch is a
+// file-scope device array; in host code its name is only a handle, so the device address is looked up
+// with cudaGetSymbolAddress once per device (under that device) and that pointer is what kernels get.
+// ------------------------------------------------------------------------------------------------
+namespace {
+static __device__ __align__(256) unsigned char g_static_scratch[CARNATOR_STATIC_SCRATCH_BYTES];
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+std::mutex g_static_mu;
+}  // namespace
+
+extern "C" carnator_status carnator_sparse_attn_static(const void* Q, const void* K, const void* V,
+                                                       const uint8_t* mask, const uint8_t* recompute_rows,
+                                                       const carnator_shape* s, void* O, float* LSE, void* stream) {
+    carnator_status st = check_shape(s, true);
+    if (st != CARNATOR_OK) return st;
+    const size_t need = carnator_attn_workspace_bytes(s);
+    if (need == 0 || need > size_t(CARNATOR_STATIC_SCRATCH_BYTES)) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error),
+                 "carnator_sparse_attn_static: this shape needs %zu bytes of scratch, the built-in array holds %zu",
+                 need, size_t(CARNATOR_STATIC_SCRATCH_BYTES));
+        return CARNATOR_ERR_WORKSPACE;
+    }
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CARNATOR_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_scratch_addr[dev]) {
+            void* p = nullptr;
+            CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));   // device address of the array on the current device
+            g_static_scratch_addr[dev] = p;
+        }
+        scratch = g_static_scratch_addr[dev];
+    }
+    // carnator_sparse_attn clears the header and rewrites every list entry it later reads.
+    return carnator_sparse_attn(Q, K, V, mask, recompute_rows, s, O, LSE, scratch, size_t(CARNATOR_STATIC_SCRATCH_BYTES), stream);
 }
 
 // ------------------------------------------------------------------------------------------------
