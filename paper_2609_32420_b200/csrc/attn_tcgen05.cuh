@@ -4,12 +4,15 @@
 // Paper: Section 3.3, "Historical Sparse-Connectivity Reuse" (only the block pairs the historical
 // structure lists are evaluated; Q, K, V are the target's own).
 //
-// Warp roles (192 threads):
+// Warp roles (224 threads):
 //   warps 0-3  softmax + epilogue; warp w owns tensor-memory lanes 32w..32w+31 = query rows
-//   warp 4     TMA producer (one lane)
+//   warp 4     TMA producer for Q and the K half tiles (one lane)
 //   warp 5     tensor-memory allocation, MMA issue (one lane)
-// Tensor memory (256 columns per CTA, two CTAs per SM): S fp32 at columns [0,128), P bf16 packed
-// into columns [0,64) once S has been read, O fp32 at columns [128,128+D).
+//   warp 6     TMA producer for the V half tiles (one lane)
+// The pipeline step is a 64-key half tile: S is double-buffered in tensor memory (columns [0,64) and
+// [64,128)), so Q K^T of step i+2 runs while the softmax warps work on step i+1 and P V of step i
+// executes; P (bf16) overwrites the first 32 columns of its own S buffer; O fp32 sits at columns
+// [128,128+D).  256 columns and <= 113 KB of shared memory per CTA: two CTAs per SM.
 // Every wait on an mbarrier is bounded; on expiry the role records CARNATOR_ERR_DEVICE_TIMEOUT in
 // the workspace header, raises a CTA-wide abort flag, and every role drains and returns.
 #pragma once
@@ -21,10 +24,13 @@
 namespace carnator {
 namespace tc {
 
-constexpr int kBlock = 128;            // query rows per CTA = keys per tile
-constexpr int kThreads = 192;
+constexpr int kBlock = 128;            // query rows per CTA = keys per listed block
+constexpr int kKeys = 64;              // keys per pipeline step (half of a block)
+constexpr int kSlots = 2;              // ring slots for K halves, V halves and S buffers
+constexpr int kThreads = 224;
+constexpr int kWarpTmaK = 4, kWarpMma = 5, kWarpTmaV = 6;
 constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColP = 0, kColO = 128;
+constexpr uint32_t kColS = 0, kColO = 128;      // S buffers at columns [0,64) and [64,128); O at [128,128+D)
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8, well inside bf16/fp32 range
 
 // ---- small PTX wrappers -----------------------------------------------------------------------
@@ -153,29 +159,29 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
     return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
 }
 
-template <int D, int STAGES>
+// Shared-memory plan.  Q: 128 x D (D/64 boxes of 128 rows x 128 B).  K and V travel as 64-key half tiles
+// (D/64 boxes of 64 rows x 128 B) through two-slot rings.
+template <int D>
 struct Cfg {
-    static constexpr int kBoxes = D / 64;                       // 64-element (128-byte) boxes per row
-    static constexpr uint32_t kBoxBytes = kBlock * 128;         // 128 rows x 128 B
-    static constexpr uint32_t kTileBytes = kBoxes * kBoxBytes;  // one 128 x D bf16 tile
+    static constexpr int kBoxes = D / 64;                           // 64-element (128-byte) boxes per row
+    static constexpr uint32_t kQBoxBytes = kBlock * 128;            // 128 rows x 128 B
+    static constexpr uint32_t kQBytes = kBoxes * kQBoxBytes;
+    static constexpr uint32_t kHBoxBytes = kKeys * 128;             // 64 rows x 128 B
+    static constexpr uint32_t kHalfBytes = kBoxes * kHBoxBytes;     // one 64 x D bf16 half tile
     static constexpr uint32_t kOffQ = 0;
-    static constexpr uint32_t kOffK = kTileBytes;
-    static constexpr uint32_t kOffV = kOffK + STAGES * kTileBytes;
-    static constexpr uint32_t kOffBar = kOffV + STAGES * kTileBytes;
-    static constexpr uint32_t kNeeded = kOffBar + 256 + 1024;   // barriers + slack to align the base to 1 KiB
+    static constexpr uint32_t kOffK = kQBytes;
+    static constexpr uint32_t kOffV = kOffK + kSlots * kHalfBytes;
+    static constexpr uint32_t kOffBar = kOffV + kSlots * kHalfBytes;
+    static constexpr uint32_t kNeeded = kOffBar + 256 + 1024;       // barriers + slack to align the base to 1 KiB
     // request enough that at most two CTAs fit an SM (two x 256 tensor-memory columns)
     static constexpr uint32_t kSmemBytes = kNeeded > 78 * 1024 ? kNeeded : 78 * 1024;
 };
 
-struct TcParams {
-    AttnArgs a;
-};
-
-template <int D, int STAGES>
+template <int D>
 __global__ void __launch_bounds__(kThreads, 2)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                     const __grid_constant__ CUtensorMap mapV, const AttnArgs a) {
-    using C = Cfg<D, STAGES>;
+    using C = Cfg<D>;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
@@ -197,35 +203,38 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         }
         return;
     }
+    // The pipeline runs on 64-key half tiles.  Every listed block gives two, except a ragged last block
+    // with at most 64 valid keys (lists ascend, so only the final entry can be the tail block).
+    const int last_valid = min(kBlock, a.N - list[count - 1] * kBlock);
+    const int T = 2 * count - (last_valid <= kKeys ? 1 : 0);
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base + C::kOffQ;
     const uint32_t sK = smem_base + C::kOffK;
     const uint32_t sV = smem_base + C::kOffV;
     const uint32_t bars = smem_base + C::kOffBar;
-    // barrier slots (8 bytes each)
-    const uint32_t bar_q = bars;
-    const uint32_t bar_s = bars + 8;
-    const uint32_t bar_p = bars + 16;
-    const uint32_t bar_o = bars + 24;
-    const uint32_t bar_drain = bars + 32;
-    auto bar_kfull = [&](int s) { return bars + 64 + 8 * s; };
-    auto bar_kempty = [&](int s) { return bars + 64 + 8 * (STAGES + s); };
-    auto bar_vfull = [&](int s) { return bars + 64 + 8 * (2 * STAGES + s); };
-    auto bar_vempty = [&](int s) { return bars + 64 + 8 * (3 * STAGES + s); };
+    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16, bar_pv = bars + 24;
+    auto bar_kfull = [&](int s) { return bars + 32 + 8 * s; };
+    auto bar_kempty = [&](int s) { return bars + 48 + 8 * s; };
+    auto bar_vfull = [&](int s) { return bars + 64 + 8 * s; };
+    auto bar_vempty = [&](int s) { return bars + 80 + 8 * s; };
+    auto bar_sfull = [&](int s) { return bars + 96 + 8 * s; };
+    auto bar_pfull = [&](int s) { return bars + 112 + 8 * s; };
     volatile int* abortp = &abort_flag;
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_s, 1); mbar_init(bar_p, kBlock); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
-        for (int s = 0; s < STAGES; ++s) {
+        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1); mbar_init(bar_pv, 1);
+        for (int s = 0; s < kSlots; ++s) {
             mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
             mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
+            mbar_init(bar_sfull(s), 1); mbar_init(bar_pfull(s), kBlock);
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 4 && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); prefetch_tmap(&mapV); }
-    if (warp == 5) {
+    if (warp == kWarpTmaK && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); }
+    if (warp == kWarpTmaV && lane == 0) prefetch_tmap(&mapV);
+    if (warp == kWarpMma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
@@ -234,79 +243,110 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (warp == 4) {
-        // ================= TMA producer =================
+    // half tile i -> (listed block, half, first key)
+    auto key0_of = [&](int i) { return list[i >> 1] * kBlock + (i & 1) * kKeys; };
+
+    if (warp == kWarpTmaK) {
+        // ================= TMA producer: Q once, then the K half tiles =================
         if (lane == 0) {
-            mbar_expect_tx(bar_q, C::kTileBytes);
+            mbar_expect_tx(bar_q, C::kQBytes);
 #pragma unroll
-            for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
-            bool ok = true;
-            int armed_k = -1, armed_v = -1;     // last tile whose loads were issued
-            for (int j = 0; j < count && ok; ++j) {
-                const int s = j % STAGES;
-                const uint32_t par = uint32_t(j / STAGES) & 1u;
-                const int J = list[j];
-                ok = mbar_wait(bar_kempty(s), par ^ 1u, abortp);
-                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, j, blockIdx.x); break; }
-                mbar_expect_tx(bar_kfull(s), C::kTileBytes);
-#pragma unroll
-                for (int x = 0; x < C::kBoxes; ++x)
-                    tma_load_4d(sK + s * C::kTileBytes + x * C::kBoxBytes, &mapK, bar_kfull(s), x * 64, J * kBlock, h, b);
-                armed_k = j;
-                ok = mbar_wait(bar_vempty(s), par ^ 1u, abortp);
-                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, j, blockIdx.x); break; }
-                mbar_expect_tx(bar_vfull(s), C::kTileBytes);
+            for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kQBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
+            int armed = -1;
+            for (int i = 0; i < T; ++i) {
+                const int s = i & 1;
+                if (!mbar_wait(bar_kempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
+                }
+                mbar_expect_tx(bar_kfull(s), C::kHalfBytes);
+                const int key0 = key0_of(i);
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
-                    tma_load_4d(sV + s * C::kTileBytes + x * C::kBoxBytes, &mapV, bar_vfull(s), x * 64, J * kBlock, h, b);
-                armed_v = j;
+                    tma_load_4d(sK + s * C::kHalfBytes + x * C::kHBoxBytes, &mapK, bar_kfull(s), x * 64, key0, h, b);
+                armed = i;
             }
-            if (*abortp) {
-                // drain: copies in flight must land before the CTA gives its shared memory back
+            if (*abortp) {      // copies in flight must land before the CTA gives its shared memory back
                 mbar_wait(bar_q, 0, abortp);
-                if (armed_k >= 0) mbar_wait(bar_kfull(armed_k % STAGES), uint32_t(armed_k / STAGES) & 1u, abortp);
-                if (armed_v >= 0) mbar_wait(bar_vfull(armed_v % STAGES), uint32_t(armed_v / STAGES) & 1u, abortp);
+                if (armed >= 0) mbar_wait(bar_kfull(armed & 1), uint32_t(armed >> 1) & 1u, abortp);
+                if (armed >= 1) mbar_wait(bar_kfull((armed - 1) & 1), uint32_t((armed - 1) >> 1) & 1u, abortp);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kWarpTmaV) {
+        // ================= TMA producer: the V half tiles =================
+        if (lane == 0) {
+            int armed = -1;
+            for (int i = 0; i < T; ++i) {
+                const int s = i & 1;
+                if (!mbar_wait(bar_vempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
+                }
+                mbar_expect_tx(bar_vfull(s), C::kHalfBytes);
+                const int key0 = key0_of(i);
+#pragma unroll
+                for (int x = 0; x < C::kBoxes; ++x)
+                    tma_load_4d(sV + s * C::kHalfBytes + x * C::kHBoxBytes, &mapV, bar_vfull(s), x * 64, key0, h, b);
+                armed = i;
+            }
+            if (*abortp) {
+                if (armed >= 0) mbar_wait(bar_vfull(armed & 1), uint32_t(armed >> 1) & 1u, abortp);
+                if (armed >= 1) mbar_wait(bar_vfull((armed - 1) & 1), uint32_t((armed - 1) >> 1) & 1u, abortp);
+            }
+        }
+    } else if (warp == kWarpMma) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(kBlock, kBlock, 0);
+            constexpr uint32_t idesc_qk = instr_desc(kBlock, kKeys, 0);
             constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
             bool ok = mbar_wait(bar_q, 0, abortp);
             if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
-            for (int j = 0; j < count && ok; ++j) {
-                const int s = j % STAGES;
-                const uint32_t par = uint32_t(j / STAGES) & 1u;
-                ok = mbar_wait(bar_kfull(s), par, abortp);
-                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, j, blockIdx.x); break; }
+            // S[i&1] = Q K_i^T : K-major operands, 16 elements of the head dimension per instruction
+            auto issue_qk = [&](int i) -> bool {
+                const int s = i & 1;
+                if (!mbar_wait(bar_kfull(s), uint32_t(i >> 1) & 1u, abortp)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, i, blockIdx.x); return false;
+                }
                 tc_fence_after();
-                // S = Q K^T : K-major operands, 16 elements of the head dimension per instruction
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
-                    mma_ss(tmem + kColS, smem_desc(sQ + off, 16, 1024), smem_desc(sK + s * C::kTileBytes + off, 16, 1024),
+                    const uint32_t inbox = (kk % 4) * 32;
+                    mma_ss(tmem + kColS + s * kKeys,
+                           smem_desc(sQ + (kk / 4) * C::kQBoxBytes + inbox, 16, 1024),
+                           smem_desc(sK + s * C::kHalfBytes + (kk / 4) * C::kHBoxBytes + inbox, 16, 1024),
                            idesc_qk, kk > 0);
                 }
-                tc_commit(bar_s);
+                tc_commit(bar_sfull(s));
                 tc_commit(bar_kempty(s));
-                ok = mbar_wait(bar_p, uint32_t(j) & 1u, abortp);
-                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, j, blockIdx.x); break; }
-                ok = mbar_wait(bar_vfull(s), par, abortp);
-                if (!ok) { set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 6, j, blockIdx.x); break; }
+                return true;
+            };
+            // O += P_i V_i : P from tensor memory (16 keys = 8 packed columns per instruction), V half tile as
+            // the MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
+            auto issue_pv = [&](int i) -> bool {
+                const int s = i & 1;
+                if (!mbar_wait(bar_pfull(s), uint32_t(i >> 1) & 1u, abortp)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, i, blockIdx.x); return false;
+                }
+                if (!mbar_wait(bar_vfull(s), uint32_t(i >> 1) & 1u, abortp)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 6, i, blockIdx.x); return false;
+                }
                 tc_fence_after();
-                // O += P V : P from tensor memory (16 keys = 8 packed columns per instruction),
-                // V tile as the MN-major B operand (rows = keys, 64-element chunks of the head dimension)
 #pragma unroll
-                for (int kk = 0; kk < kBlock / 16; ++kk) {
-                    mma_ts(tmem + kColO, tmem + kColP + kk * 8,
-                           smem_desc(sV + s * C::kTileBytes + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (j > 0) || (kk > 0));
+                for (int kk = 0; kk < kKeys / 16; ++kk) {
+                    mma_ts(tmem + kColO, tmem + kColS + s * kKeys + kk * 8,
+                           smem_desc(sV + s * C::kHalfBytes + kk * 2048, C::kHBoxBytes, 1024), idesc_pv, (i > 0) || (kk > 0));
                 }
                 tc_commit(bar_vempty(s));
-                if (j == count - 1) tc_commit(bar_o);
+                tc_commit(bar_pv);
+                return true;
+            };
+            if (ok) ok = issue_qk(0);
+            if (ok && T > 1) ok = issue_qk(1);
+            for (int i = 0; i < T && ok; ++i) {
+                ok = issue_pv(i);
+                // S[i&1] is free again once P_i V_i has been queued (MMAs of one thread execute in order)
+                if (ok && i + 2 < T) ok = issue_qk(i + 2);
             }
-            if (*abortp) {
-                // make sure no MMA is still running before tensor memory is released
+            if (ok) tc_commit(bar_o);
+            if (*abortp) {      // make sure no MMA is still running before tensor memory is released
                 tc_commit(bar_drain);
                 mbar_wait(bar_drain, 0, abortp);
             }
@@ -317,36 +357,41 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         const int row = q0 + tid;
         float m_used = -INFINITY, l_sum = 0.f;
         bool ok = true;
-        for (int j = 0; j < count; ++j) {
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_s, uint32_t(j) & 1u, abortp));   // warp-uniform: the loads below are collective
-            if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, j, blockIdx.x); break; }
+        for (int i = 0; i < T; ++i) {
+            const int sb = i & 1;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull(sb), uint32_t(i >> 1) & 1u, abortp));   // warp-uniform: the loads below are collective
+            if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, i, blockIdx.x); break; }
             tc_fence_after();
-            const int J = list[j];
-            const int nvalid = min(kBlock, a.N - J * kBlock);
-            float s[4][32];
-#pragma unroll
-            for (int c = 0; c < 4; ++c) tmem_ld32(tmem + lane_base + kColS + c * 32, s[c]);
+            const int nvalid = a.N - key0_of(i);          // >= 1 by construction of T
+            const uint32_t tS = tmem + lane_base + kColS + sb * kKeys;
+            float s[2][32];
+            tmem_ld32(tS, s[0]);
+            tmem_ld32(tS + 32, s[1]);
             tmem_wait_ld();
-            if (nvalid < kBlock) {               // ragged last key block (warp-uniform): keys >= N never count
+            if (nvalid < kKeys) {                // ragged tail (warp-uniform): keys >= N never count
 #pragma unroll
-                for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 2; ++c)
 #pragma unroll
-                    for (int i = 0; i < 32; ++i)
-                        if (c * 32 + i >= nvalid) s[c][i] = -INFINITY;
+                    for (int e = 0; e < 32; ++e)
+                        if (c * 32 + e >= nvalid) s[c][e] = -INFINITY;
             }
             // row maximum of the raw scores (the scale is positive), four independent chains
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+            for (int c = 0; c < 2; ++c)
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx4[i & 3] = fmaxf(mx4[i & 3], s[c][i]);
+                for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], s[c][e]);
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
             // lazy rescale: the reference maximum only moves when it would grow by more than the threshold
             const bool grow = (mx > m_used + kRescaleThreshold);
-            if (j == 0) {
+            if (i == 0) {
                 m_used = mx;
             } else if (__any_sync(0xffffffffu, grow)) {
-                // s_full(j) was committed after P V of tile j-1, so O is quiescent here
+                // O must be quiescent: wait until P V of half tile i-1 has completed (P V of tile i cannot start
+                // before this warp has delivered P_i)
+                ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, uint32_t(i - 1) & 1u, abortp));
+                if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 9, i, blockIdx.x); break; }
+                tc_fence_after();
                 const float m_new = grow ? mx : m_used;
                 const float f = ex2_approx(m_used - m_new);
 #pragma unroll
@@ -356,37 +401,36 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                     tmem_wait_ld();
                     uint32_t r[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(o[i] * f);
+                    for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(o[e] * f);
                     tmem_st32(tmem + lane_base + kColO + c * 32, r);
                 }
                 l_sum *= f;
                 m_used = m_new;
             }
-            // P = exp2(s * scale - m_used): one FFMA + one MUFU per element, packed to bf16 pairs in columns [0,64)
+            // P = exp2(s * scale - m_used): one FFMA + one MUFU per element, packed bf16 pairs over S's own columns
             const float neg_m = -m_used;
             float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 uint32_t pk[16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float p0 = ex2_approx(fmaf(s[c][2 * i], a.scale_log2, neg_m));
-                    const float p1 = ex2_approx(fmaf(s[c][2 * i + 1], a.scale_log2, neg_m));
-                    part[i & 1] += p0;
-                    part[2 + (i & 1)] += p1;
-                    pk[i] = pack_bf16(p0, p1);
+                for (int e = 0; e < 16; ++e) {
+                    const float p0 = ex2_approx(fmaf(s[c][2 * e], a.scale_log2, neg_m));
+                    const float p1 = ex2_approx(fmaf(s[c][2 * e + 1], a.scale_log2, neg_m));
+                    part[e & 1] += p0;
+                    part[2 + (e & 1)] += p1;
+                    pk[e] = pack_bf16(p0, p1);
                 }
-                tmem_st16(tmem + lane_base + kColP + c * 16, pk);
+                tmem_st16(tS + c * 16, pk);
             }
-            const float part_sum = (part[0] + part[1]) + (part[2] + part[3]);
-            l_sum += part_sum;
+            l_sum += (part[0] + part[1]) + (part[2] + part[3]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_p);
+            mbar_arrive(bar_pfull(sb));
         }
         if (ok) {
             ok = __all_sync(0xffffffffu, mbar_wait(bar_o, 0, abortp));
-            if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 8, count, blockIdx.x);
+            if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 8, T, blockIdx.x);
         }
         if (ok) {
             tc_fence_after();
@@ -415,7 +459,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kWarpMma) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
@@ -442,9 +486,9 @@ inline EncodeTiledFn encode_fn() {
     return fn;
 }
 
-// 4-D map over a [B,H,N,D] bf16 tensor with arbitrary (16-byte multiple) strides: box = 64 x 128 x 1 x 1,
+// 4-D map over a [B,H,N,D] bf16 tensor with arbitrary (16-byte multiple) strides: box = 64 x box_rows x 1 x 1,
 // 128-byte swizzle, rows >= N read as zero.
-inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, int D, const int64_t st[3]) {
+inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, int D, const int64_t st[3], int box_rows) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(N), cuuint64_t(H), cuuint64_t(B)};
@@ -455,7 +499,7 @@ inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, in
     if (s_h == 0) s_h = row * N;
     if (s_b == 0) s_b = s_h * H;
     cuuint64_t strides[3] = {row, s_h, s_b};
-    cuuint32_t box[4] = {64, cuuint32_t(kBlock), 1, 1};
+    cuuint32_t box[4] = {64, cuuint32_t(box_rows), 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, estr,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -469,11 +513,11 @@ inline bool tcgen05_supported(const carnator_shape* s) {
     return s->block_q == tc::kBlock && s->block_k == tc::kBlock && (s->D == 64 || s->D == 128);
 }
 
-template <int D, int STAGES>
+template <int D>
 inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
                                  cudaStream_t stream, char* err, size_t errlen) {
-    using C = tc::Cfg<D, STAGES>;
-    auto kern = tc::attn_tcgen05_kernel<D, STAGES>;
+    using C = tc::Cfg<D>;
+    auto kern = tc::attn_tcgen05_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmemBytes));
     if (e != cudaSuccess) { snprintf(err, errlen, "cudaFuncSetAttribute(tcgen05): %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
     dim3 grid(a.nqb, a.H, a.B);
@@ -486,13 +530,14 @@ inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const
 inline carnator_status launch_tcgen05(const AttnArgs& a, const carnator_shape* s, cudaStream_t stream,
                                       char* err, size_t errlen, long long* launches) {
     CUtensorMap mq, mk, mv;
-    if (!tc::make_map(&mq, a.Q, a.B, a.H, a.N, s->D, a.qs) || !tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks) ||
-        !tc::make_map(&mv, a.V, a.B, a.H, a.N, s->D, a.vs)) {
+    if (!tc::make_map(&mq, a.Q, a.B, a.H, a.N, s->D, a.qs, tc::kBlock) ||
+        !tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks, tc::kKeys) ||
+        !tc::make_map(&mv, a.V, a.B, a.H, a.N, s->D, a.vs, tc::kKeys)) {
         snprintf(err, errlen, "cuTensorMapEncodeTiled failed or is unavailable");
         return CARNATOR_ERR_CUDA;
     }
-    carnator_status st = (s->D == 128) ? launch_tc<128, 1>(a, mq, mk, mv, stream, err, errlen)
-                                       : launch_tc<64, 2>(a, mq, mk, mv, stream, err, errlen);
+    carnator_status st = (s->D == 128) ? launch_tc<128>(a, mq, mk, mv, stream, err, errlen)
+                                       : launch_tc<64>(a, mq, mk, mv, stream, err, errlen);
     if (st == CARNATOR_OK) *launches = 1;
     return st;
 }
