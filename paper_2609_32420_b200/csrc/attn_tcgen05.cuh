@@ -58,10 +58,11 @@ __device__ __forceinline__ unsigned long long global_ns() {
     return t;
 }
 // Bounded wait: gives up after ~2 s (or when another role has aborted) and raises the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0) {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 0; it < (1u << 30); ++it) {
+        if (sleep_ns) __nanosleep(sleep_ns);
         if (mbar_try(bar, parity)) return true;
         if ((it & 255u) == 255u) {
             if (*abort_flag) return false;
@@ -255,7 +256,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             int armed = -1;
             for (int i = 0; i < T; ++i) {
                 const int s = i & 1;
-                if (!mbar_wait(bar_kempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp)) {
+                if (!mbar_wait(bar_kempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
                 }
                 mbar_expect_tx(bar_kfull(s), C::kHalfBytes);
@@ -277,7 +278,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             int armed = -1;
             for (int i = 0; i < T; ++i) {
                 const int s = i & 1;
-                if (!mbar_wait(bar_vempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp)) {
+                if (!mbar_wait(bar_vempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
                 }
                 mbar_expect_tx(bar_vfull(s), C::kHalfBytes);
@@ -322,7 +323,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             // the MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
             auto issue_pv = [&](int i) -> bool {
                 const int s = i & 1;
-                if (!mbar_wait(bar_pfull(s), uint32_t(i >> 1) & 1u, abortp)) {
+                if (!mbar_wait(bar_pfull(s), uint32_t(i >> 1) & 1u, abortp, 40)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, i, blockIdx.x); return false;
                 }
                 if (!mbar_wait(bar_vfull(s), uint32_t(i >> 1) & 1u, abortp)) {
@@ -359,7 +360,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         bool ok = true;
         for (int i = 0; i < T; ++i) {
             const int sb = i & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull(sb), uint32_t(i >> 1) & 1u, abortp));   // warp-uniform: the loads below are collective
+            ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull(sb), uint32_t(i >> 1) & 1u, abortp, 20));   // warp-uniform: the loads below are collective
             if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, i, blockIdx.x); break; }
             tc_fence_after();
             const int nvalid = a.N - key0_of(i);          // >= 1 by construction of T
