@@ -4,15 +4,15 @@
 // Paper: Section 3.3, "Historical Sparse-Connectivity Reuse" (only the block pairs the historical
 // structure lists are evaluated; Q, K, V are the target's own).
 //
-// Warp roles (224 threads):
-//   warps 0-3  softmax + epilogue; warp w owns tensor-memory lanes 32w..32w+31 = query rows
-//   warp 4     TMA producer for Q and the K half tiles (one lane)
-//   warp 5     tensor-memory allocation, MMA issue (one lane)
-//   warp 6     TMA producer for the V half tiles (one lane)
-// The pipeline step is a 64-key half tile: S is double-buffered in tensor memory (columns [0,64) and
-// [64,128)), so Q K^T of step i+2 runs while the softmax warps work on step i+1 and P V of step i
-// executes; P (bf16) overwrites the first 32 columns of its own S buffer; O fp32 sits at columns
-// [128,128+D).  256 columns and <= 113 KB of shared memory per CTA: two CTAs per SM.
+// Warp roles (352 threads, one CTA per SM):
+//   warps 0-3  softmax group 0, warps 4-7 softmax group 1: the groups take the 128-key steps in turn; within
+//              a group warp w owns tensor-memory lanes 32w..32w+31 = query rows.  Both also run the epilogue.
+//   warp 8     TMA producer for Q and the K tiles (one lane)
+//   warp 9     tensor-memory allocation, MMA issue (one lane)
+//   warp 10    TMA producer for the V tiles (one lane)
+// Tensor memory (512 columns): three score buffers S0 | S1 | S2 (128 fp32 columns each) and O (D columns).
+// Q K^T of step i+2 is issued as soon as P V of step i-1 is queued, so two score tiles are always ahead of the
+// softmax groups; P (bf16) overwrites the first 64 columns of its own score buffer.
 // Every wait on an mbarrier is bounded; on expiry the role records CARNATOR_ERR_DEVICE_TIMEOUT in
 // the workspace header, raises a CTA-wide abort flag, and every role drains and returns.
 #pragma once
@@ -24,13 +24,13 @@
 namespace carnator {
 namespace tc {
 
-constexpr int kBlock = 128;            // query rows per CTA = keys per listed block
-constexpr int kKeys = 64;              // keys per pipeline step (half of a block)
-constexpr int kSlots = 2;              // ring slots for K halves, V halves and S buffers
-constexpr int kThreads = 224;
-constexpr int kWarpTmaK = 4, kWarpMma = 5, kWarpTmaV = 6;
-constexpr int kTmemCols = 256;
-constexpr uint32_t kColS = 0, kColO = 128;      // S buffers at columns [0,64) and [64,128); O at [128,128+D)
+constexpr int kBlock = 128;            // query rows per CTA = keys per step
+constexpr int kSBufs = 3;              // score buffers in tensor memory
+constexpr int kStages = 2;             // ring slots for K tiles and for V tiles
+constexpr int kSoftmaxWarps = 8;       // two warpgroups taking the steps in turn
+constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
+constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
+constexpr int kTmemCols = 512;         // S0 | S1 | S2 | O
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8, well inside bf16/fp32 range
 
 // ---- small PTX wrappers -----------------------------------------------------------------------
@@ -71,6 +71,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
     *abort_flag = 1;
     return false;
+}
+
+// Warp-collective form: lane 0 waits (bounded), the outcome is broadcast; the shuffle orders the other
+// lanes' later reads after lane 0's acquire.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0) {
+    int ok = 1;
+    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, sleep_ns) ? 1 : 0;
+    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+}
+// One arrival per warp once every lane's earlier writes are ordered before it.
+__device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(bar);
 }
 
 __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar,
@@ -160,42 +173,41 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
     return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
 }
 
-// Shared-memory plan.  Q: 128 x D (D/64 boxes of 128 rows x 128 B).  K and V travel as 64-key half tiles
-// (D/64 boxes of 64 rows x 128 B) through two-slot rings.
+// Shared-memory plan.  Q, and every K / V tile, is 128 rows x D held as D/64 boxes of 128 rows x 128 B
+// (128-byte swizzle).  K and V tiles travel through kStages-slot rings.
 template <int D>
 struct Cfg {
-    static constexpr int kBoxes = D / 64;                           // 64-element (128-byte) boxes per row
-    static constexpr uint32_t kQBoxBytes = kBlock * 128;            // 128 rows x 128 B
-    static constexpr uint32_t kQBytes = kBoxes * kQBoxBytes;
-    static constexpr uint32_t kHBoxBytes = kKeys * 128;             // 64 rows x 128 B
-    static constexpr uint32_t kHalfBytes = kBoxes * kHBoxBytes;     // one 64 x D bf16 half tile
+    static constexpr int kBoxes = D / 64;
+    static constexpr uint32_t kBoxBytes = kBlock * 128;             // 128 rows x 128 B
+    static constexpr uint32_t kTileBytes = kBoxes * kBoxBytes;      // one 128 x D bf16 tile
     static constexpr uint32_t kOffQ = 0;
-    static constexpr uint32_t kOffK = kQBytes;
-    static constexpr uint32_t kOffV = kOffK + kSlots * kHalfBytes;
-    static constexpr uint32_t kOffBar = kOffV + kSlots * kHalfBytes;
-    static constexpr uint32_t kNeeded = kOffBar + 256 + 1024;       // barriers + slack to align the base to 1 KiB
-    // request enough that at most two CTAs fit an SM (two x 256 tensor-memory columns)
-    static constexpr uint32_t kSmemBytes = kNeeded > 78 * 1024 ? kNeeded : 78 * 1024;
+    static constexpr uint32_t kOffK = kTileBytes;
+    static constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
+    static constexpr uint32_t kOffBar = kOffV + kStages * kTileBytes;
+    static constexpr uint32_t kSmemBytes = kOffBar + 512 + 1024;    // barriers + slack to align the base to 1 KiB
+    static constexpr uint32_t kColO = kSBufs * kBlock;              // O accumulator after the S buffers
 };
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                     const __grid_constant__ CUtensorMap mapV, const AttnArgs a) {
     using C = Cfg<D>;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    __shared__ float r_pub[kSBufs][kBlock];     // reference maximum after step i, slot i % 3 (handed from one warpgroup to the other)
+    __shared__ float fin[2][2][kBlock];         // per warpgroup: final reference maximum and partial row sum
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.z, h = blockIdx.y;
     const int64_t bh = int64_t(b) * a.H + h;
     const int I = a.order[bh * a.nqb + blockIdx.x];
-    const int count = a.counts[bh * a.nqb + I];
+    const int T = a.counts[bh * a.nqb + I];           // steps = listed key blocks
     const int32_t* list = a.lists + (bh * a.nqb + I) * int64_t(a.nkb);
     const int q0 = I * kBlock;
 
-    if (count == 0) {                       // nothing to attend to: O = 0, LSE = -inf
+    if (T == 0) {                           // nothing to attend to: O = 0, LSE = -inf
         if (tid < kBlock && q0 + tid < a.N) {
             __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(q0 + tid) * a.os[2];
 #pragma unroll
@@ -204,33 +216,37 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         }
         return;
     }
-    // The pipeline runs on 64-key half tiles.  Every listed block gives two, except a ragged last block
-    // with at most 64 valid keys (lists ascend, so only the final entry can be the tail block).
-    const int last_valid = min(kBlock, a.N - list[count - 1] * kBlock);
-    const int T = 2 * count - (last_valid <= kKeys ? 1 : 0);
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
     const uint32_t sQ = smem_base + C::kOffQ;
     const uint32_t sK = smem_base + C::kOffK;
     const uint32_t sV = smem_base + C::kOffV;
     const uint32_t bars = smem_base + C::kOffBar;
-    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16, bar_pv = bars + 24;
-    auto bar_kfull = [&](int s) { return bars + 32 + 8 * s; };
-    auto bar_kempty = [&](int s) { return bars + 48 + 8 * s; };
-    auto bar_vfull = [&](int s) { return bars + 64 + 8 * s; };
-    auto bar_vempty = [&](int s) { return bars + 80 + 8 * s; };
-    auto bar_sfull = [&](int s) { return bars + 96 + 8 * s; };
-    auto bar_pfull = [&](int s) { return bars + 112 + 8 * s; };
+    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16;
+    auto bar_kfull = [&](int s) { return bars + 32 + 8 * s; };       // up to 4 stages each
+    auto bar_kempty = [&](int s) { return bars + 64 + 8 * s; };
+    auto bar_vfull = [&](int s) { return bars + 96 + 8 * s; };
+    auto bar_vempty = [&](int s) { return bars + 128 + 8 * s; };
+    auto bar_sfull = [&](int s) { return bars + 160 + 8 * s; };      // 3 S buffers
+    auto bar_pfull = [&](int s) { return bars + 192 + 8 * s; };
+    auto bar_ref = [&](int s, int q) { return bars + 224 + 8 * (s * 4 + q); };   // r_pub slot s, lane quarter q
+    auto bar_fin = [&](int q) { return bars + 320 + 8 * q; };
+    auto bar_pvdone = [&](int s) { return bars + 352 + 8 * s; };     // P V of the step that used score buffer s has completed
     volatile int* abortp = &abort_flag;
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1); mbar_init(bar_pv, 1);
-        for (int s = 0; s < kSlots; ++s) {
+        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
+        for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
             mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
-            mbar_init(bar_sfull(s), 1); mbar_init(bar_pfull(s), kBlock);
         }
+        for (int s = 0; s < kSBufs; ++s) {
+            mbar_init(bar_sfull(s), 1); mbar_init(bar_pvdone(s), 1);
+            mbar_init(bar_pfull(s), 4);                                      // one arrival per softmax warp of the group
+            for (int q = 0; q < 4; ++q) mbar_init(bar_ref(s, q), 1);
+        }
+        for (int q = 0; q < 4; ++q) mbar_init(bar_fin(q), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kWarpTmaK && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); }
@@ -244,107 +260,104 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    // half tile i -> (listed block, half, first key)
-    auto key0_of = [&](int i) { return list[i >> 1] * kBlock + (i & 1) * kKeys; };
-
     if (warp == kWarpTmaK) {
-        // ================= TMA producer: Q once, then the K half tiles =================
+        // ================= TMA producer: Q once, then the K tiles =================
         if (lane == 0) {
-            mbar_expect_tx(bar_q, C::kQBytes);
+            mbar_expect_tx(bar_q, C::kTileBytes);
 #pragma unroll
-            for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kQBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
+            for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
             int armed = -1;
             for (int i = 0; i < T; ++i) {
-                const int s = i & 1;
-                if (!mbar_wait(bar_kempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp, 200)) {
+                const int s = i % kStages;
+                if (!mbar_wait(bar_kempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
                 }
-                mbar_expect_tx(bar_kfull(s), C::kHalfBytes);
-                const int key0 = key0_of(i);
+                mbar_expect_tx(bar_kfull(s), C::kTileBytes);
+                const int key0 = list[i] * kBlock;
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
-                    tma_load_4d(sK + s * C::kHalfBytes + x * C::kHBoxBytes, &mapK, bar_kfull(s), x * 64, key0, h, b);
+                    tma_load_4d(sK + s * C::kTileBytes + x * C::kBoxBytes, &mapK, bar_kfull(s), x * 64, key0, h, b);
                 armed = i;
             }
             if (*abortp) {      // copies in flight must land before the CTA gives its shared memory back
                 mbar_wait(bar_q, 0, abortp);
-                if (armed >= 0) mbar_wait(bar_kfull(armed & 1), uint32_t(armed >> 1) & 1u, abortp);
-                if (armed >= 1) mbar_wait(bar_kfull((armed - 1) & 1), uint32_t((armed - 1) >> 1) & 1u, abortp);
+                for (int k = 0; k < kStages && armed - k >= 0; ++k)
+                    mbar_wait(bar_kfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, abortp);
             }
         }
     } else if (warp == kWarpTmaV) {
-        // ================= TMA producer: the V half tiles =================
+        // ================= TMA producer: the V tiles =================
         if (lane == 0) {
             int armed = -1;
             for (int i = 0; i < T; ++i) {
-                const int s = i & 1;
-                if (!mbar_wait(bar_vempty(s), (uint32_t(i >> 1) & 1u) ^ 1u, abortp, 200)) {
+                const int s = i % kStages;
+                if (!mbar_wait(bar_vempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
                 }
-                mbar_expect_tx(bar_vfull(s), C::kHalfBytes);
-                const int key0 = key0_of(i);
+                mbar_expect_tx(bar_vfull(s), C::kTileBytes);
+                const int key0 = list[i] * kBlock;
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
-                    tma_load_4d(sV + s * C::kHalfBytes + x * C::kHBoxBytes, &mapV, bar_vfull(s), x * 64, key0, h, b);
+                    tma_load_4d(sV + s * C::kTileBytes + x * C::kBoxBytes, &mapV, bar_vfull(s), x * 64, key0, h, b);
                 armed = i;
             }
             if (*abortp) {
-                if (armed >= 0) mbar_wait(bar_vfull(armed & 1), uint32_t(armed >> 1) & 1u, abortp);
-                if (armed >= 1) mbar_wait(bar_vfull((armed - 1) & 1), uint32_t((armed - 1) >> 1) & 1u, abortp);
+                for (int k = 0; k < kStages && armed - k >= 0; ++k)
+                    mbar_wait(bar_vfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, abortp);
             }
         }
     } else if (warp == kWarpMma) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            constexpr uint32_t idesc_qk = instr_desc(kBlock, kKeys, 0);
+            constexpr uint32_t idesc_qk = instr_desc(kBlock, kBlock, 0);
             constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
             bool ok = mbar_wait(bar_q, 0, abortp);
             if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
-            // S[i&1] = Q K_i^T : K-major operands, 16 elements of the head dimension per instruction
+            // S[i % 3] = Q K_i^T : K-major operands, 16 elements of the head dimension per instruction
             auto issue_qk = [&](int i) -> bool {
-                const int s = i & 1;
-                if (!mbar_wait(bar_kfull(s), uint32_t(i >> 1) & 1u, abortp)) {
+                const int s = i % kStages, sb = i % kSBufs;
+                if (!mbar_wait(bar_kfull(s), uint32_t(i / kStages) & 1u, abortp, 20)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, i, blockIdx.x); return false;
                 }
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t inbox = (kk % 4) * 32;
-                    mma_ss(tmem + kColS + s * kKeys,
-                           smem_desc(sQ + (kk / 4) * C::kQBoxBytes + inbox, 16, 1024),
-                           smem_desc(sK + s * C::kHalfBytes + (kk / 4) * C::kHBoxBytes + inbox, 16, 1024),
-                           idesc_qk, kk > 0);
+                    const uint32_t off = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
+                    mma_ss(tmem + sb * kBlock, smem_desc(sQ + off, 16, 1024),
+                           smem_desc(sK + s * C::kTileBytes + off, 16, 1024), idesc_qk, kk > 0);
                 }
-                tc_commit(bar_sfull(s));
+                tc_commit(bar_sfull(sb));
                 tc_commit(bar_kempty(s));
                 return true;
             };
-            // O += P_i V_i : P from tensor memory (16 keys = 8 packed columns per instruction), V half tile as
-            // the MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
+            // O += P_i V_i : P from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
+            // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
             auto issue_pv = [&](int i) -> bool {
-                const int s = i & 1;
-                if (!mbar_wait(bar_pfull(s), uint32_t(i >> 1) & 1u, abortp, 40)) {
+                const int s = i % kStages, sb = i % kSBufs;
+                if (!mbar_wait(bar_pfull(sb), uint32_t(i / kSBufs) & 1u, abortp, 20)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, i, blockIdx.x); return false;
                 }
-                if (!mbar_wait(bar_vfull(s), uint32_t(i >> 1) & 1u, abortp)) {
+                if (!mbar_wait(bar_vfull(s), uint32_t(i / kStages) & 1u, abortp, 20)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 6, i, blockIdx.x); return false;
                 }
                 tc_fence_after();
 #pragma unroll
-                for (int kk = 0; kk < kKeys / 16; ++kk) {
-                    mma_ts(tmem + kColO, tmem + kColS + s * kKeys + kk * 8,
-                           smem_desc(sV + s * C::kHalfBytes + kk * 2048, C::kHBoxBytes, 1024), idesc_pv, (i > 0) || (kk > 0));
+                for (int kk = 0; kk < kBlock / 16; ++kk) {
+                    mma_ts(tmem + C::kColO, tmem + sb * kBlock + kk * 8,
+                           smem_desc(sV + s * C::kTileBytes + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (i > 0) || (kk > 0));
                 }
                 tc_commit(bar_vempty(s));
-                tc_commit(bar_pv);
+                tc_commit(bar_pvdone(sb));
                 return true;
             };
-            if (ok) ok = issue_qk(0);
-            if (ok && T > 1) ok = issue_qk(1);
+            // kSBufs score tiles are in flight: K slots free up as soon as their Q K^T has run, so the K ring
+            // does not limit how far the scores run ahead of the softmax groups
+            constexpr int kAhead = kSBufs;
+            for (int i = 0; i < kAhead && i < T && ok; ++i) ok = issue_qk(i);
             for (int i = 0; i < T && ok; ++i) {
                 ok = issue_pv(i);
-                // S[i&1] is free again once P_i V_i has been queued (MMAs of one thread execute in order)
-                if (ok && i + 2 < T) ok = issue_qk(i + 2);
+                // S[i % 3] and K slot are free again once P_i V_i has been queued (MMAs of one thread execute in order)
+                if (ok && i + kAhead < T) ok = issue_qk(i + kAhead);
             }
             if (ok) tc_commit(bar_o);
             if (*abortp) {      // make sure no MMA is still running before tensor memory is released
@@ -353,25 +366,34 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
         }
     } else {
-        // ================= softmax + epilogue (warps 0-3) =================
-        const uint32_t lane_base = uint32_t(warp * 32) << 16;
-        const int row = q0 + tid;
-        float m_used = -INFINITY, l_sum = 0.f;
+        // ================= softmax + epilogue (warps 0-7) =================
+        // Two warpgroups take the steps in turn (group g: steps g, g+2, ...), each with one warp per
+        // tensor-memory lane quarter, so one group's exponentials run while the other group's scores are
+        // being produced.  Both feed the same O accumulator, so they share one reference maximum per row:
+        // the group that handles step i derives R_i from R_{i-1} (published by the other group right after
+        // its row-maximum pass) and publishes R_i in turn.  The reference only moves when a row maximum
+        // exceeds it by more than the threshold; then this group rescales O before delivering P_i.
+        const int quarter = warp & 3, wg = warp >> 2;
+        const int r_loc = quarter * 32 + lane;                      // query row within the tile
+        const uint32_t lane_base = uint32_t(quarter * 32) << 16;
+        const int row = q0 + r_loc;
+        float m_w = -INFINITY, l_w = 0.f;                           // this group's reference and partial row sum
         bool ok = true;
-        for (int i = 0; i < T; ++i) {
-            const int sb = i & 1;
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_sfull(sb), uint32_t(i >> 1) & 1u, abortp, 20));   // warp-uniform: the loads below are collective
+        for (int i = wg; i < T; i += 2) {
+            const int sb = i % kSBufs;
+            const uint32_t sph = uint32_t(i / kSBufs) & 1u;
+            ok = mbar_wait_warp(bar_sfull(sb), sph, abortp, 20);   // warp-uniform: the loads below are collective
             if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, i, blockIdx.x); break; }
             tc_fence_after();
-            const int nvalid = a.N - key0_of(i);          // >= 1 by construction of T
-            const uint32_t tS = tmem + lane_base + kColS + sb * kKeys;
-            float s[2][32];
-            tmem_ld32(tS, s[0]);
-            tmem_ld32(tS + 32, s[1]);
-            tmem_wait_ld();
-            if (nvalid < kKeys) {                // ragged tail (warp-uniform): keys >= N never count
+            const int nvalid = a.N - list[i] * kBlock;              // >= 1; < 128 only for a ragged last block
+            const uint32_t tS = tmem + lane_base + sb * kBlock;
+            float s[4][32];
 #pragma unroll
-                for (int c = 0; c < 2; ++c)
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
+            tmem_wait_ld();
+            if (nvalid < kBlock) {               // ragged tail (warp-uniform): keys >= N never count
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int e = 0; e < 32; ++e)
                         if (c * 32 + e >= nvalid) s[c][e] = -INFINITY;
@@ -379,40 +401,48 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             // row maximum of the raw scores (the scale is positive), four independent chains
             float mx4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-            for (int c = 0; c < 2; ++c)
+            for (int c = 0; c < 4; ++c)
 #pragma unroll
                 for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], s[c][e]);
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
-            // lazy rescale: the reference maximum only moves when it would grow by more than the threshold
-            const bool grow = (mx > m_used + kRescaleThreshold);
-            if (i == 0) {
-                m_used = mx;
-            } else if (__any_sync(0xffffffffu, grow)) {
-                // O must be quiescent: wait until P V of half tile i-1 has completed (P V of tile i cannot start
-                // before this warp has delivered P_i)
-                ok = __all_sync(0xffffffffu, mbar_wait(bar_pv, uint32_t(i - 1) & 1u, abortp));
+            // reference handed over from step i-1
+            float r_prev = -INFINITY, r_now = mx;
+            bool grow = false;
+            if (i > 0) {
+                ok = mbar_wait_warp(bar_ref((i - 1) % kSBufs, quarter), uint32_t((i - 1) / kSBufs) & 1u, abortp, 0);
+                if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 10, i, blockIdx.x); break; }
+                r_prev = r_pub[(i - 1) % kSBufs][r_loc];
+                grow = mx > r_prev + kRescaleThreshold;
+                r_now = grow ? mx : r_prev;
+            }
+            r_pub[sb][r_loc] = r_now;
+            mbar_arrive_warp(bar_ref(sb, quarter));
+            if (i > 0 && __any_sync(0xffffffffu, grow)) {
+                // O must be quiescent: P V of step i-1 complete (P V of step i cannot start before this group
+                // delivers P_i; a rescale by the other group for step i+1 waits for P V of step i).  One barrier
+                // per score buffer keeps the phase unambiguous: S_i being ready implies P V of step i-3, and
+                // with it the previous use of this barrier (step i-4), is complete.
+                ok = mbar_wait_warp(bar_pvdone((i - 1) % kSBufs), uint32_t((i - 1) / kSBufs) & 1u, abortp, 0);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 9, i, blockIdx.x); break; }
                 tc_fence_after();
-                const float m_new = grow ? mx : m_used;
-                const float f = ex2_approx(m_used - m_new);
+                const float f = ex2_approx(r_prev - r_now);          // 1 for rows that did not move
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     float o[32];
-                    tmem_ld32(tmem + lane_base + kColO + c * 32, o);
+                    tmem_ld32(tmem + lane_base + C::kColO + c * 32, o);
                     tmem_wait_ld();
                     uint32_t r[32];
 #pragma unroll
                     for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(o[e] * f);
-                    tmem_st32(tmem + lane_base + kColO + c * 32, r);
+                    tmem_st32(tmem + lane_base + C::kColO + c * 32, r);
                 }
-                l_sum *= f;
-                m_used = m_new;
             }
-            // P = exp2(s * scale - m_used): one FFMA + one MUFU per element, packed bf16 pairs over S's own columns
-            const float neg_m = -m_used;
+            if (m_w != r_now) { l_w *= ex2_approx(m_w - r_now); m_w = r_now; }   // first use: l_w = 0, exp2(-inf) = 0
+            // P = exp2(s * scale - R_i): one FFMA + one MUFU per element, packed bf16 pairs over S's own columns
+            const float neg_m = -r_now;
             float part[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
@@ -424,23 +454,35 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 }
                 tmem_st16(tS + c * 16, pk);
             }
-            l_sum += (part[0] + part[1]) + (part[2] + part[3]);
+            l_w += (part[0] + part[1]) + (part[2] + part[3]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar_pfull(sb));
+            mbar_arrive_warp(bar_pfull(sb));
+        }
+        // combine the two groups' sums under the final reference (the later step holds the larger one)
+        if (ok) {
+            fin[wg][0][r_loc] = m_w;
+            fin[wg][1][r_loc] = l_w;
+            mbar_arrive_warp(bar_fin(quarter));
+            ok = mbar_wait_warp(bar_fin(quarter), 0, abortp, 0);
+            if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 11, T, blockIdx.x);
         }
         if (ok) {
-            ok = __all_sync(0xffffffffu, mbar_wait(bar_o, 0, abortp));
+            ok = mbar_wait_warp(bar_o, 0, abortp, 20);
             if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 8, T, blockIdx.x);
         }
         if (ok) {
             tc_fence_after();
-            const float inv = 1.f / l_sum;
-            __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(row) * a.os[2];
+            const float m0 = fin[0][0][r_loc], m1 = fin[1][0][r_loc];
+            const float r_fin = fmaxf(m0, m1);
+            const float l_tot = fin[0][1][r_loc] * ex2_approx(m0 - r_fin) + fin[1][1][r_loc] * ex2_approx(m1 - r_fin);
+            const float inv = 1.f / l_tot;
+            // each group writes half of the head dimension
+            __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(row) * a.os[2] + wg * (D / 2);
 #pragma unroll
-            for (int c = 0; c < D / 32; ++c) {
+            for (int c = 0; c < D / 64; ++c) {
                 float o[32];
-                tmem_ld32(tmem + lane_base + kColO + c * 32, o);      // warp-collective: every lane takes part
+                tmem_ld32(tmem + lane_base + C::kColO + wg * (D / 2) + c * 32, o);      // warp-collective: every lane takes part
                 tmem_wait_ld();
                 if (row < a.N) {
 #pragma unroll
@@ -454,7 +496,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                     }
                 }
             }
-            if (row < a.N) a.LSE[bh * a.N + row] = (m_used + log2f(l_sum)) * kLn2;
+            if (wg == 0 && row < a.N) a.LSE[bh * a.N + row] = (r_fin + log2f(l_tot)) * kLn2;
         }
     }
 
@@ -532,8 +574,8 @@ inline carnator_status launch_tcgen05(const AttnArgs& a, const carnator_shape* s
                                       char* err, size_t errlen, long long* launches) {
     CUtensorMap mq, mk, mv;
     if (!tc::make_map(&mq, a.Q, a.B, a.H, a.N, s->D, a.qs, tc::kBlock) ||
-        !tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks, tc::kKeys) ||
-        !tc::make_map(&mv, a.V, a.B, a.H, a.N, s->D, a.vs, tc::kKeys)) {
+        !tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks, tc::kBlock) ||
+        !tc::make_map(&mv, a.V, a.B, a.H, a.N, s->D, a.vs, tc::kBlock)) {
         snprintf(err, errlen, "cuTensorMapEncodeTiled failed or is unavailable");
         return CARNATOR_ERR_CUDA;
     }
