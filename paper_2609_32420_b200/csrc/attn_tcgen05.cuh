@@ -10,9 +10,9 @@
 //   warp 8     TMA producer for Q and the K tiles (one lane)
 //   warp 9     tensor-memory allocation, MMA issue (one lane)
 //   warp 10    TMA producer for the V tiles (one lane)
-// Tensor memory (512 columns): three score buffers S0 | S1 | S2 (128 fp32 columns each) and O (D columns).
-// Q K^T of step i+2 is issued as soon as P V of step i-1 is queued, so two score tiles are always ahead of the
-// softmax groups; P (bf16) overwrites the first 64 columns of its own score buffer.
+// Tensor memory (512 columns): S0 | S1 (128 fp32 columns each, one per softmax group), P0 | P1 (64 columns
+// of packed bf16 each), O (D fp32 columns).  A group signals as soon as it has pulled its scores into
+// registers, so Q K^T of its next step runs underneath its own exponentials; P V is issued in step order.
 // Every wait on an mbarrier is bounded; on expiry the role records CARNATOR_ERR_DEVICE_TIMEOUT in
 // the workspace header, raises a CTA-wide abort flag, and every role drains and returns.
 #pragma once
@@ -25,12 +25,15 @@ namespace carnator {
 namespace tc {
 
 constexpr int kBlock = 128;            // query rows per CTA = keys per step
-constexpr int kSBufs = 3;              // score buffers in tensor memory
+constexpr int kSBufs = 2;              // score buffers in tensor memory, one per softmax group
+constexpr int kRefSlots = 3;           // hand-over slots of the shared reference maximum
 constexpr int kStages = 2;             // ring slots for K tiles and for V tiles
 constexpr int kSoftmaxWarps = 8;       // two warpgroups taking the steps in turn
 constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
 constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
-constexpr int kTmemCols = 512;         // S0 | S1 | S2 | O
+constexpr int kTmemCols = 512;         // S0 | S1 | P0 | P1 | O
+constexpr uint32_t kColP = 2 * kBlock; // packed bf16 probabilities: 64 columns per group
+constexpr uint32_t kColO = 2 * kBlock + 2 * 64;
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8, well inside bf16/fp32 range
 
 // ---- small PTX wrappers -----------------------------------------------------------------------
@@ -185,7 +188,6 @@ struct Cfg {
     static constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
     static constexpr uint32_t kOffBar = kOffV + kStages * kTileBytes;
     static constexpr uint32_t kSmemBytes = kOffBar + 512 + 1024;    // barriers + slack to align the base to 1 KiB
-    static constexpr uint32_t kColO = kSBufs * kBlock;              // O accumulator after the S buffers
 };
 
 template <int D>
@@ -196,7 +198,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float r_pub[kSBufs][kBlock];     // reference maximum after step i, slot i % 3 (handed from one warpgroup to the other)
+    __shared__ float r_pub[kRefSlots][kBlock];     // reference maximum after step i, slot i % 3 (handed from one warpgroup to the other)
     __shared__ float fin[2][2][kBlock];         // per warpgroup: final reference maximum and partial row sum
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -227,8 +229,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     auto bar_kempty = [&](int s) { return bars + 64 + 8 * s; };
     auto bar_vfull = [&](int s) { return bars + 96 + 8 * s; };
     auto bar_vempty = [&](int s) { return bars + 128 + 8 * s; };
-    auto bar_sfull = [&](int s) { return bars + 160 + 8 * s; };      // 3 S buffers
-    auto bar_pfull = [&](int s) { return bars + 192 + 8 * s; };
+    auto bar_sfull = [&](int s) { return bars + 160 + 8 * s; };      // S_g holds fresh scores
+    auto bar_sfree = [&](int s) { return bars + 176 + 8 * s; };      // group g has read S_g into registers
+    auto bar_pfull = [&](int s) { return bars + 192 + 8 * s; };      // P_g is complete
     auto bar_ref = [&](int s, int q) { return bars + 224 + 8 * (s * 4 + q); };   // r_pub slot s, lane quarter q
     auto bar_fin = [&](int q) { return bars + 320 + 8 * q; };
     auto bar_pvdone = [&](int s) { return bars + 352 + 8 * s; };     // P V of the step that used score buffer s has completed
@@ -243,9 +246,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         }
         for (int s = 0; s < kSBufs; ++s) {
             mbar_init(bar_sfull(s), 1); mbar_init(bar_pvdone(s), 1);
-            mbar_init(bar_pfull(s), 4);                                      // one arrival per softmax warp of the group
-            for (int q = 0; q < 4; ++q) mbar_init(bar_ref(s, q), 1);
+            mbar_init(bar_pfull(s), 4); mbar_init(bar_sfree(s), 4);          // one arrival per softmax warp of the group
         }
+        for (int s = 0; s < kRefSlots; ++s)
+            for (int q = 0; q < 4; ++q) mbar_init(bar_ref(s, q), 1);
         for (int q = 0; q < 4; ++q) mbar_init(bar_fin(q), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -313,9 +317,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
             bool ok = mbar_wait(bar_q, 0, abortp);
             if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
-            // S[i % 3] = Q K_i^T : K-major operands, 16 elements of the head dimension per instruction
+            // S_g = Q K_i^T (g = i & 1): K-major operands, 16 elements of the head dimension per instruction
             auto issue_qk = [&](int i) -> bool {
-                const int s = i % kStages, sb = i % kSBufs;
+                const int s = i % kStages, g = i & 1;
                 if (!mbar_wait(bar_kfull(s), uint32_t(i / kStages) & 1u, abortp, 20)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, i, blockIdx.x); return false;
                 }
@@ -323,41 +327,52 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
                 for (int kk = 0; kk < D / 16; ++kk) {
                     const uint32_t off = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
-                    mma_ss(tmem + sb * kBlock, smem_desc(sQ + off, 16, 1024),
+                    mma_ss(tmem + g * kBlock, smem_desc(sQ + off, 16, 1024),
                            smem_desc(sK + s * C::kTileBytes + off, 16, 1024), idesc_qk, kk > 0);
                 }
-                tc_commit(bar_sfull(sb));
+                tc_commit(bar_sfull(g));
                 tc_commit(bar_kempty(s));
                 return true;
             };
-            // O += P_i V_i : P from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
+            // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
             // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
             auto issue_pv = [&](int i) -> bool {
-                const int s = i % kStages, sb = i % kSBufs;
-                if (!mbar_wait(bar_pfull(sb), uint32_t(i / kSBufs) & 1u, abortp, 20)) {
-                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, i, blockIdx.x); return false;
-                }
+                const int s = i % kStages, g = i & 1;
                 if (!mbar_wait(bar_vfull(s), uint32_t(i / kStages) & 1u, abortp, 20)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 6, i, blockIdx.x); return false;
                 }
                 tc_fence_after();
 #pragma unroll
                 for (int kk = 0; kk < kBlock / 16; ++kk) {
-                    mma_ts(tmem + C::kColO, tmem + sb * kBlock + kk * 8,
+                    mma_ts(tmem + kColO, tmem + kColP + g * 64 + kk * 8,
                            smem_desc(sV + s * C::kTileBytes + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (i > 0) || (kk > 0));
                 }
                 tc_commit(bar_vempty(s));
-                tc_commit(bar_pvdone(sb));
+                tc_commit(bar_pvdone(g));
                 return true;
             };
-            // kSBufs score tiles are in flight: K slots free up as soon as their Q K^T has run, so the K ring
-            // does not limit how far the scores run ahead of the softmax groups
-            constexpr int kAhead = kSBufs;
-            for (int i = 0; i < kAhead && i < T && ok; ++i) ok = issue_qk(i);
-            for (int i = 0; i < T && ok; ++i) {
-                ok = issue_pv(i);
-                // S[i % 3] and K slot are free again once P_i V_i has been queued (MMAs of one thread execute in order)
-                if (ok && i + kAhead < T) ok = issue_qk(i + kAhead);
+            // Q K^T of step i+2 may go as soon as group g has pulled S_g (step i) into registers; P V of step i
+            // goes, in step order, once P_g is complete.  Whichever is ready first is issued first.
+            int qk_next = 0, pv_next = 0;
+            for (; qk_next < 2 && qk_next < T && ok; ++qk_next) ok = issue_qk(qk_next);
+            unsigned long long t_last = global_ns();     // time of the last issued batch
+            uint32_t idle = 0;
+            while (pv_next < T && ok) {
+                bool progress = false;
+                if (qk_next < T && mbar_try(bar_sfree(qk_next & 1), uint32_t((qk_next - 2) >> 1) & 1u)) {
+                    ok = issue_qk(qk_next); ++qk_next; progress = true;
+                }
+                if (ok && mbar_try(bar_pfull(pv_next & 1), uint32_t(pv_next >> 1) & 1u)) {
+                    ok = issue_pv(pv_next); ++pv_next; progress = true;
+                }
+                if (progress) { idle = 0; t_last = global_ns(); continue; }
+                __nanosleep(20);
+                if ((++idle & 1023u) == 0) {         // bounded: ~2 s without any progress, or another role aborted
+                    if (*abortp) { ok = false; break; }
+                    if (idle >= (1u << 28) || global_ns() - t_last > 2000000000ull) {
+                        *abortp = 1; set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, pv_next, blockIdx.x); ok = false; break;
+                    }
+                }
             }
             if (ok) tc_commit(bar_o);
             if (*abortp) {      // make sure no MMA is still running before tensor memory is released
@@ -380,17 +395,20 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         float m_w = -INFINITY, l_w = 0.f;                           // this group's reference and partial row sum
         bool ok = true;
         for (int i = wg; i < T; i += 2) {
-            const int sb = i % kSBufs;
-            const uint32_t sph = uint32_t(i / kSBufs) & 1u;
-            ok = mbar_wait_warp(bar_sfull(sb), sph, abortp, 20);   // warp-uniform: the loads below are collective
+            const int rs = i % kRefSlots;
+            const uint32_t sph = uint32_t(i >> 1) & 1u;
+            ok = mbar_wait_warp(bar_sfull(wg), sph, abortp, 20);   // warp-uniform: the loads below are collective
             if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, i, blockIdx.x); break; }
             tc_fence_after();
             const int nvalid = a.N - list[i] * kBlock;              // >= 1; < 128 only for a ragged last block
-            const uint32_t tS = tmem + lane_base + sb * kBlock;
+            const uint32_t tS = tmem + lane_base + wg * kBlock;
+            const uint32_t tP = tmem + lane_base + kColP + wg * 64;
             float s[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
             tmem_wait_ld();
+            tc_fence_before();
+            mbar_arrive_warp(bar_sfree(wg));     // the scores are in registers: S_g may take the scores of step i+2
             if (nvalid < kBlock) {               // ragged tail (warp-uniform): keys >= N never count
 #pragma unroll
                 for (int c = 0; c < 4; ++c)
@@ -409,32 +427,37 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             float r_prev = -INFINITY, r_now = mx;
             bool grow = false;
             if (i > 0) {
-                ok = mbar_wait_warp(bar_ref((i - 1) % kSBufs, quarter), uint32_t((i - 1) / kSBufs) & 1u, abortp, 0);
+                ok = mbar_wait_warp(bar_ref((i - 1) % kRefSlots, quarter), uint32_t((i - 1) / kRefSlots) & 1u, abortp, 0);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 10, i, blockIdx.x); break; }
-                r_prev = r_pub[(i - 1) % kSBufs][r_loc];
+                r_prev = r_pub[(i - 1) % kRefSlots][r_loc];
                 grow = mx > r_prev + kRescaleThreshold;
                 r_now = grow ? mx : r_prev;
             }
-            r_pub[sb][r_loc] = r_now;
-            mbar_arrive_warp(bar_ref(sb, quarter));
+            r_pub[rs][r_loc] = r_now;
+            mbar_arrive_warp(bar_ref(rs, quarter));
+            // P_g is free again once P V of this group's previous step (i-2) has completed; in-order execution
+            // then also covers P V of step i-3
+            if (i >= 2) {
+                ok = mbar_wait_warp(bar_pvdone(wg), uint32_t((i - 2) >> 1) & 1u, abortp, 0);
+                if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 12, i, blockIdx.x); break; }
+            }
             if (i > 0 && __any_sync(0xffffffffu, grow)) {
-                // O must be quiescent: P V of step i-1 complete (P V of step i cannot start before this group
-                // delivers P_i; a rescale by the other group for step i+1 waits for P V of step i).  One barrier
-                // per score buffer keeps the phase unambiguous: S_i being ready implies P V of step i-3, and
-                // with it the previous use of this barrier (step i-4), is complete.
-                ok = mbar_wait_warp(bar_pvdone((i - 1) % kSBufs), uint32_t((i - 1) / kSBufs) & 1u, abortp, 0);
+                // O must be quiescent: P V of step i-1 (the other group's) complete.  P V is issued in step order
+                // and that of step i cannot start before this group delivers P_i; the wait above has already
+                // established that P V of step i-3 is complete, so the phase of this barrier is unambiguous.
+                ok = mbar_wait_warp(bar_pvdone(wg ^ 1), uint32_t((i - 1) >> 1) & 1u, abortp, 0);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 9, i, blockIdx.x); break; }
                 tc_fence_after();
                 const float f = ex2_approx(r_prev - r_now);          // 1 for rows that did not move
 #pragma unroll
                 for (int c = 0; c < D / 32; ++c) {
                     float o[32];
-                    tmem_ld32(tmem + lane_base + C::kColO + c * 32, o);
+                    tmem_ld32(tmem + lane_base + kColO + c * 32, o);
                     tmem_wait_ld();
                     uint32_t r[32];
 #pragma unroll
                     for (int e = 0; e < 32; ++e) r[e] = __float_as_uint(o[e] * f);
-                    tmem_st32(tmem + lane_base + C::kColO + c * 32, r);
+                    tmem_st32(tmem + lane_base + kColO + c * 32, r);
                 }
             }
             if (m_w != r_now) { l_w *= ex2_approx(m_w - r_now); m_w = r_now; }   // first use: l_w = 0, exp2(-inf) = 0
@@ -452,12 +475,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                     part[2 + (e & 1)] += p1;
                     pk[e] = pack_bf16(p0, p1);
                 }
-                tmem_st16(tS + c * 16, pk);
+                tmem_st16(tP + c * 16, pk);
             }
             l_w += (part[0] + part[1]) + (part[2] + part[3]);
             tmem_wait_st();
             tc_fence_before();
-            mbar_arrive_warp(bar_pfull(sb));
+            mbar_arrive_warp(bar_pfull(wg));
         }
         // combine the two groups' sums under the final reference (the later step holds the larger one)
         if (ok) {
@@ -482,7 +505,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
             for (int c = 0; c < D / 64; ++c) {
                 float o[32];
-                tmem_ld32(tmem + lane_base + C::kColO + wg * (D / 2) + c * 32, o);      // warp-collective: every lane takes part
+                tmem_ld32(tmem + lane_base + kColO + wg * (D / 2) + c * 32, o);      // warp-collective: every lane takes part
                 tmem_wait_ld();
                 if (row < a.N) {
 #pragma unroll
