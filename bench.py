@@ -371,13 +371,13 @@ def run_ours(args):
     # ---- roofline of the dominant kernel -----------------------------------------------------------
     attn_tflops = flops / (ms_attn * 1e-3) / 1e12
     traffic = None
-    tpath = os.path.join(ROOT, "profiles", "traffic.json")
+    tpath = os.path.join(ROOT, "profiles", "attn_traffic.txt")
     if os.path.exists(tpath):
-        with open(tpath) as f:
-            tj = json.load(f)
-        ent = tj.get(w.name)
-        if ent and ent.get("tiles"):
-            traffic = ent["dram_bytes_per_launch"] * tiles / ent["tiles"]
+        base = w.name.split("[")[0]
+        for ln in open(tpath):
+            parts = ln.split()
+            if len(parts) == 3 and parts[0] == base and int(parts[2]) > 0:
+                traffic = float(parts[1]) * tiles / float(parts[2])
     roofline = {"bound": "tensor", "kernel": "sparse attention", "achieved": attn_tflops, "peak": peaks["bf16"],
                 "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16"], "traffic": traffic,
                 "peak_source": peaks["source"] + " bf16_tflops (burst)", "frac_of_sustained": attn_tflops / peaks["bf16_sustained"],
