@@ -302,4 +302,71 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
     for (int J = tid; J < a.nkb; J += nt) a.mask[row + J] = keep[J];
 }
 
+// Top-k mode without a sort: one warp per (b,h,I).  Each lane keeps the order-preserving keys of the
+// blocks J = lane, lane+32, ... in registers; the k-th largest key is found bit by bit (largest T with
+// #(key >= T) >= k), then equal keys are admitted in ascending block order until k is reached.
+template <int NPL>   // keys per lane: nkb <= 32 * NPL
+__global__ void __launch_bounds__(256) select_topk_kernel(SelectArgs a, int rows) {
+    const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int lane = threadIdx.x & 31;
+    if (warp >= rows) return;
+    const int I = warp % a.nqb;
+    const int64_t row = int64_t(warp) * a.nkb;
+    const float* s = a.scores + row;
+
+    uint32_t key[NPL];
+    uint32_t forced_bits[(NPL + 31) / 32];
+#pragma unroll
+    for (int w = 0; w < (NPL + 31) / 32; ++w) forced_bits[w] = 0u;
+    int my_forced = 0;
+#pragma unroll
+    for (int t = 0; t < NPL; ++t) {
+        const int J = t * 32 + lane;
+        uint32_t k = 0u;                       // always-kept and out-of-range entries never compete
+        if (J < a.nkb) {
+            if (forced_block(I, J, a.g)) { forced_bits[t >> 5] |= 1u << (t & 31); ++my_forced; }
+            else k = ordered_bits(s[J]);
+        }
+        key[t] = k;
+    }
+    int nforced = my_forced;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) nforced += __shfl_xor_sync(0xffffffffu, nforced, o);
+    const int nfree = a.nkb - nforced;
+    int n_admit = a.count_includes_forced ? max(0, a.k_all - nforced) : topk_count_dev(a.keep_ratio, nfree);
+    n_admit = min(n_admit, nfree);
+
+    uint32_t T = 0xFFFFFFFFu;                  // nothing admitted by score
+    int need_eq = 0;
+    if (n_admit > 0) {
+        T = 0u;
+        for (int bit = 31; bit >= 0; --bit) {
+            const uint32_t cand = T | (1u << bit);
+            int c = 0;
+#pragma unroll
+            for (int t = 0; t < NPL; ++t) c += (key[t] >= cand) ? 1 : 0;
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+            if (c >= n_admit) T = cand;
+        }
+        int gt = 0;
+#pragma unroll
+        for (int t = 0; t < NPL; ++t) gt += (key[t] > T) ? 1 : 0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) gt += __shfl_xor_sync(0xffffffffu, gt, o);
+        need_eq = n_admit - gt;                // >= 1 blocks with key == T, lowest block index first
+    }
+    int seen_eq = 0;
+#pragma unroll
+    for (int t = 0; t < NPL; ++t) {
+        const int J = t * 32 + lane;
+        const bool eq = (n_admit > 0) && key[t] == T;
+        const unsigned bal = __ballot_sync(0xffffffffu, eq);
+        const int rank = seen_eq + __popc(bal & ((1u << lane) - 1u));
+        seen_eq += __popc(bal);
+        const bool keep = ((forced_bits[t >> 5] >> (t & 31)) & 1u) || (n_admit > 0 && key[t] > T) || (eq && rank < need_eq);
+        if (J < a.nkb) a.mask[row + J] = keep ? 1 : 0;
+    }
+}
+
 }  // namespace carnator

@@ -173,11 +173,21 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
         sa.k_all = topk_count_host(p->keep_ratio, nkb);
         sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
         sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
-        size_t smem = size_t(sa.npad) * 8 * (p->mode == CARNATOR_MODE_CUMMASS ? 2 : 1) + ((nkb + 15) & ~15);
-        st = allow_smem(select_kernel, 72 * 1024);
-        if (st != CARNATOR_OK) return st;
-        dim3 grid(nqb, s->H, s->B);
-        select_kernel<<<grid, 256, smem, stream>>>(sa);
+        if (p->mode == CARNATOR_MODE_TOPK) {
+            // register-resident selection, one warp per row
+            const int rows = s->B * s->H * nqb;
+            const int grid = ceil_div(rows, 8);
+            if (nkb <= 32 * 8) select_topk_kernel<8><<<grid, 256, 0, stream>>>(sa, rows);
+            else if (nkb <= 32 * 32) select_topk_kernel<32><<<grid, 256, 0, stream>>>(sa, rows);
+            else select_topk_kernel<128><<<grid, 256, 0, stream>>>(sa, rows);
+        } else {
+            // cumulative-mass mode needs the sorted order: shared-memory bitonic sort, one CTA per row
+            size_t smem = size_t(sa.npad) * 8 * 2 + ((nkb + 15) & ~15);
+            st = allow_smem(select_kernel, 72 * 1024);
+            if (st != CARNATOR_OK) return st;
+            dim3 grid(nqb, s->H, s->B);
+            select_kernel<<<grid, 256, smem, stream>>>(sa);
+        }
         LAUNCH_CHECK("select_kernel");
     }
     return CARNATOR_OK;
