@@ -4,12 +4,14 @@
 // Paper: Section 3.3, "Historical Sparse-Connectivity Reuse" (only the block pairs the historical
 // structure lists are evaluated; Q, K, V are the target's own).
 //
-// Warp roles (352 threads, one CTA per SM):
+// Warp roles (384 threads = three warpgroups, one CTA per SM):
 //   warps 0-3  softmax group 0, warps 4-7 softmax group 1: the groups take the 128-key steps in turn; within
 //              a group warp w owns tensor-memory lanes 32w..32w+31 = query rows.  Both also run the epilogue.
 //   warp 8     TMA producer for Q and the K tiles (one lane)
 //   warp 9     tensor-memory allocation, MMA issue (one lane)
-//   warp 10    TMA producer for the V tiles (one lane)
+//   warp 10    TMA producer for the V tiles (one lane); warp 11 idles
+// The third warpgroup gives most of its registers to the softmax groups (setmaxnreg), which hold a full
+// 128-column score row per thread.
 // Tensor memory (512 columns): S0 | S1 (128 fp32 columns each, one per softmax group), P0 | P1 (64 columns
 // of packed bf16 each), O (D fp32 columns).  A group signals as soon as it has pulled its scores into
 // registers, so Q K^T of its next step runs underneath its own exponentials; P V is issued in step order.
@@ -29,7 +31,7 @@ constexpr int kSBufs = 2;              // score buffers in tensor memory, one pe
 constexpr int kRefSlots = 3;           // hand-over slots of the shared reference maximum
 constexpr int kStages = 2;             // ring slots for K tiles and for V tiles
 constexpr int kSoftmaxWarps = 8;       // two warpgroups taking the steps in turn
-constexpr int kThreads = (kSoftmaxWarps + 3) * 32;
+constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // third warpgroup: two TMA producers, the MMA issuer, one idle warp
 constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
 constexpr int kTmemCols = 512;         // S0 | S1 | P0 | P1 | O
 constexpr uint32_t kColP = 2 * kBlock; // packed bf16 probabilities: 64 columns per group
@@ -264,6 +266,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
+    if (warp >= kSoftmaxWarps) {
+    // Register budget: the producer / MMA warpgroup needs few registers and hands the rest to the softmax groups.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
     if (warp == kWarpTmaK) {
         // ================= TMA producer: Q once, then the K tiles =================
         if (lane == 0) {
@@ -380,7 +385,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 mbar_wait(bar_drain, 0, abortp);
             }
         }
+    }
     } else {
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory");
         // ================= softmax + epilogue (warps 0-7) =================
         // Two warpgroups take the steps in turn (group g: steps g, g+2, ...), each with one warp per
         // tensor-memory lane quarter, so one group's exponentials run while the other group's scores are
