@@ -12,6 +12,16 @@ def widen(bits):
     return wl.bf16_bits_to_f32(bits).astype(np.float64)
 
 
+def record(kind, what, **values):
+    """Append one line of measured parity errors to the file named by CARNATOR_PARITY_LOG (if set)."""
+    import json
+    import os
+    path = os.environ.get("CARNATOR_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps({"kind": kind, "case": what, **values}) + "\n")
+
+
 # tolerances the GPU path must meet against the oracle
 O_MAX_ABS = 2e-2
 O_MEAN_ABS = 2e-3
@@ -36,7 +46,9 @@ def check_attention(O_gpu, LSE_gpu, O_ref, LSE_ref, what=""):
     fin = okl & ~ninf
     rel = np.abs(L_gpu[fin] - L_ref[fin]) / np.maximum(np.abs(L_ref[fin]), 1.0)
     assert rel.max(initial=0.0) <= LSE_REL, f"{what}: LSE rel {rel.max()}"
-    return float(err.max(initial=0.0)), float(err.mean() if err.size else 0.0), float(rel.max(initial=0.0))
+    out = float(err.max(initial=0.0)), float(err.mean() if err.size else 0.0), float(rel.max(initial=0.0))
+    record("attention", what, o_max_abs=out[0], o_mean_abs=out[1], lse_rel=out[2], n_values=int(err.size))
+    return out
 
 
 def check_mask(mask_gpu, mask_ref, scores_ref, theta_ref, forced, topk_mode=True, what=""):
@@ -46,6 +58,7 @@ def check_mask(mask_gpu, mask_ref, scores_ref, theta_ref, forced, topk_mode=True
     mask_ref = np.asarray(mask_ref) != 0
     diff = mask_gpu != mask_ref
     n_diff = int(diff.sum())
+    record("mask", what, mismatches=n_diff, blocks=int(mask_ref.size), density=float(mask_ref.mean()))
     if n_diff == 0:
         return 0
     B, H, nqb, nkb = mask_ref.shape

@@ -141,10 +141,11 @@ def test_strided_inputs_and_rows_past_n_untouched(impl):
     check_attention(o_to_host(O[:, :, :N]), L.cpu().numpy(), O_ref, L_ref, "strided")
 
 
-FULL = [("wan1p3b_480p", None), ("cogvideox5b", None), ("wan14b_720p", None), ("hunyuan_720p", 0.10)]
+FULL = [("wan1p3b_480p", None), ("cogvideox5b", None), ("wan14b_720p", None), ("hunyuan_720p", 0.10),
+        ("hunyuan_720p", 1.00)]      # keep ratio 1.0: all-ones mask, the dense check
 
 
-@pytest.mark.parametrize("name,density", FULL, ids=[f[0] for f in FULL])
+@pytest.mark.parametrize("name,density", FULL, ids=[f[0] + ("" if f[1] is None else f"_{f[1]}") for f in FULL])
 def test_full_size_workload_sampled_rows(name, density):
     """Whole layer at the benchmark's launch configuration (mask from the GPU builder on the
     historical Q/K pair); sampled (head, query block) rows against the oracle."""
@@ -166,6 +167,8 @@ def test_full_size_workload_sampled_rows(name, density):
     Qb, Kb, Vb = wl.gen_qkv(w, heads=heads)
     O_ref, L_ref = orc.attention_rows(Qb, Kb, Vb, w.N, w.block, w.block, w.scale, mask, rec, rows)
     O_g, L_g = gather_rows(O, L, rows, w)
-    check_attention(O_g, L_g, O_ref, L_ref, name)
+    check_attention(O_g, L_g, O_ref, L_ref, f"{name} keep={w.build.keep_ratio}")
+    if density == 1.0:
+        assert bool((mask_dev == 1).all())
     # properties that hold at any size: every valid row finite, no row past N touched is checked above by shape
     assert torch.isfinite(O.float()).all() and torch.isfinite(L).all()
