@@ -8,8 +8,9 @@
 //   warps 0-3  softmax group 0, warps 4-7 softmax group 1: the groups take the 128-key steps in turn; within
 //              a group warp w owns tensor-memory lanes 32w..32w+31 = query rows.  Both also run the epilogue.
 //   warp 8     TMA producer for Q and the K tiles (one lane)
-//   warp 9     tensor-memory allocation, MMA issue (one lane)
-//   warp 10    TMA producer for the V tiles (one lane); warp 11 idles
+//   warp 9     tensor-memory allocation, issue of the Q K^T batches (one lane)
+//   warp 10    TMA producer for the V tiles (one lane)
+//   warp 11    issue of the P V batches (one lane)
 // The third warpgroup gives most of its registers to the softmax groups (setmaxnreg), which hold a full
 // 128-column score row per thread.
 // Tensor memory (512 columns): S0 | S1 (128 fp32 columns each, one per softmax group), P0 | P1 (64 columns
@@ -32,7 +33,7 @@ constexpr int kRefSlots = 3;           // hand-over slots of the shared referenc
 constexpr int kStages = 2;             // ring slots for K tiles and for V tiles
 constexpr int kSoftmaxWarps = 8;       // two warpgroups taking the steps in turn
 constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // third warpgroup: two TMA producers, the MMA issuer, one idle warp
-constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
+constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10, kWarpMmaPV = 11;
 constexpr int kTmemCols = 512;         // S0 | S1 | P0 | P1 | O
 constexpr uint32_t kColP = 2 * kBlock; // packed bf16 probabilities: 64 columns per group
 constexpr uint32_t kColO = 2 * kBlock + 2 * 64;
@@ -226,7 +227,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     const uint32_t sK = smem_base + C::kOffK;
     const uint32_t sV = smem_base + C::kOffV;
     const uint32_t bars = smem_base + C::kOffBar;
-    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16;
+    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16, bar_drain2 = bars + 24;
     auto bar_kfull = [&](int s) { return bars + 32 + 8 * s; };       // up to 4 stages each
     auto bar_kempty = [&](int s) { return bars + 64 + 8 * s; };
     auto bar_vfull = [&](int s) { return bars + 96 + 8 * s; };
@@ -241,7 +242,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
+        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1); mbar_init(bar_drain2, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
             mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
@@ -316,10 +317,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
         }
     } else if (warp == kWarpMma) {
-        // ================= MMA issuer =================
+        // ================= MMA issuers =================
+        // Two issuing threads: warp 9 queues the Q K^T batches, warp 11 the P V batches.  The two chains touch
+        // disjoint tensor-memory columns (S_g vs P_g and O), so neither has to wait behind the other's queue.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kBlock, kBlock, 0);
-            constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
             bool ok = mbar_wait(bar_q, 0, abortp);
             if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
             // S_g = Q K_i^T (g = i & 1): K-major operands, 16 elements of the head dimension per instruction
@@ -339,6 +341,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 tc_commit(bar_kempty(s));
                 return true;
             };
+            // Q K^T of step i may go as soon as group g has pulled S_g of step i-2 into registers
+            for (int i = 0; i < T && ok; ++i) {
+                if (i >= 2 && !mbar_wait(bar_sfree(i & 1), uint32_t((i - 2) >> 1) & 1u, abortp, 20)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 14, i, blockIdx.x); ok = false; break;
+                }
+                ok = issue_qk(i);
+            }
+            if (*abortp) {      // make sure no MMA of this thread is still running before tensor memory is released
+                tc_commit(bar_drain);
+                mbar_wait(bar_drain, 0, abortp);
+            }
+        }
+    } else if (warp == kWarpMmaPV) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
+            bool ok = true;
             // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
             // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
             auto issue_pv = [&](int i) -> bool {
@@ -356,33 +374,17 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 tc_commit(bar_pvdone(g));
                 return true;
             };
-            // Q K^T of step i+2 may go as soon as group g has pulled S_g (step i) into registers; P V of step i
-            // goes, in step order, once P_g is complete.  Whichever is ready first is issued first.
-            int qk_next = 0, pv_next = 0;
-            for (; qk_next < 2 && qk_next < T && ok; ++qk_next) ok = issue_qk(qk_next);
-            unsigned long long t_last = global_ns();     // time of the last issued batch
-            uint32_t idle = 0;
-            while (pv_next < T && ok) {
-                bool progress = false;
-                if (qk_next < T && mbar_try(bar_sfree(qk_next & 1), uint32_t((qk_next - 2) >> 1) & 1u)) {
-                    ok = issue_qk(qk_next); ++qk_next; progress = true;
+            // P V in step order, each once P_g is complete
+            for (int i = 0; i < T && ok; ++i) {
+                if (!mbar_wait(bar_pfull(i & 1), uint32_t(i >> 1) & 1u, abortp, 20)) {
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, i, blockIdx.x); ok = false; break;
                 }
-                if (ok && mbar_try(bar_pfull(pv_next & 1), uint32_t(pv_next >> 1) & 1u)) {
-                    ok = issue_pv(pv_next); ++pv_next; progress = true;
-                }
-                if (progress) { idle = 0; t_last = global_ns(); continue; }
-                __nanosleep(20);
-                if ((++idle & 1023u) == 0) {         // bounded: ~2 s without any progress, or another role aborted
-                    if (*abortp) { ok = false; break; }
-                    if (idle >= (1u << 28) || global_ns() - t_last > 2000000000ull) {
-                        *abortp = 1; set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, pv_next, blockIdx.x); ok = false; break;
-                    }
-                }
+                ok = issue_pv(i);
             }
             if (ok) tc_commit(bar_o);
-            if (*abortp) {      // make sure no MMA is still running before tensor memory is released
-                tc_commit(bar_drain);
-                mbar_wait(bar_drain, 0, abortp);
+            if (*abortp) {
+                tc_commit(bar_drain2);
+                mbar_wait(bar_drain2, 0, abortp);
             }
         }
     }
