@@ -180,7 +180,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
 }
 
 // Shared-memory plan.  Q, and every K / V tile, is 128 rows x D held as D/64 boxes of 128 rows x 128 B
-// (128-byte swizzle).  K and V tiles travel through kStages-slot rings.
+// (128-byte swizzle).  K and V tiles travel through kStages-slot rings (separate rings, separate producers).
 template <int D>
 struct Cfg {
     static constexpr int kBoxes = D / 64;
