@@ -307,12 +307,34 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
 // #(key >= T) >= k), then equal keys are admitted in ascending block order until k is reached.
 template <int NPL>   // keys per lane: nkb <= 32 * NPL
 __global__ void __launch_bounds__(256) select_topk_kernel(SelectArgs a, int rows) {
+    // frame span of every key block, computed once per CTA (two integer divisions per block)
+    extern __shared__ int2 kframes[];
+    const Geometry g = a.g;
+    for (int J = threadIdx.x; J < a.nkb; J += blockDim.x) {
+        const int k_lo = max(J * g.bk, g.n_text), k_hi = min(g.N, (J + 1) * g.bk) - 1;
+        kframes[J] = (k_hi >= k_lo) ? make_int2((k_lo - g.n_text) / g.hw, (k_hi - g.n_text) / g.hw) : make_int2(1, 0);
+    }
+    __syncthreads();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp >= rows) return;
     const int I = warp % a.nqb;
     const int64_t row = int64_t(warp) * a.nkb;
     const float* s = a.scores + row;
+
+    // the query block's side of the always-kept rule
+    const bool text_row = g.text_dense && g.n_text > 0 && I * g.bq < g.n_text;
+    const int text_cols = (g.text_dense && g.n_text > 0) ? (g.n_text + g.bk - 1) / g.bk : 0;   // key blocks holding text
+    int f_lo = 0, f_hi = 0;
+    bool has_window = false;                   // the query block holds video tokens and a window is asked for
+    if (g.window >= 0) {
+        const int q_lo = max(I * g.bq, g.n_text), q_hi = min(g.N, (I + 1) * g.bq) - 1;
+        if (q_hi >= q_lo) {
+            has_window = true;
+            f_lo = max(0, (q_lo - g.n_text) / g.hw - g.window);
+            f_hi = min(g.T - 1, (q_hi - g.n_text) / g.hw + g.window);
+        }
+    }
 
     uint32_t key[NPL];
     uint32_t forced_bits[(NPL + 31) / 32];
@@ -324,7 +346,9 @@ __global__ void __launch_bounds__(256) select_topk_kernel(SelectArgs a, int rows
         const int J = t * 32 + lane;
         uint32_t k = 0u;                       // always-kept and out-of-range entries never compete
         if (J < a.nkb) {
-            if (forced_block(I, J, a.g)) { forced_bits[t >> 5] |= 1u << (t & 31); ++my_forced; }
+            const int2 kf = kframes[J];
+            const bool forced = text_row || J < text_cols || (has_window && kf.x <= kf.y && kf.x <= f_hi && kf.y >= f_lo);
+            if (forced) { forced_bits[t >> 5] |= 1u << (t & 31); ++my_forced; }
             else k = ordered_bits(s[J]);
         }
         key[t] = k;

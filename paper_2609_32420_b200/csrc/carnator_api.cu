@@ -177,9 +177,11 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
             // register-resident selection, one warp per row
             const int rows = s->B * s->H * nqb;
             const int grid = ceil_div(rows, 8);
-            if (nkb <= 32 * 8) select_topk_kernel<8><<<grid, 256, 0, stream>>>(sa, rows);
-            else if (nkb <= 32 * 32) select_topk_kernel<32><<<grid, 256, 0, stream>>>(sa, rows);
-            else select_topk_kernel<128><<<grid, 256, 0, stream>>>(sa, rows);
+            const size_t tbl = size_t(nkb) * sizeof(int2);     // key-block frame table (<= 32 KiB)
+            if (nkb <= 32 * 8) select_topk_kernel<8><<<grid, 256, tbl, stream>>>(sa, rows);
+            else if (nkb <= 32 * 20) select_topk_kernel<20><<<grid, 256, tbl, stream>>>(sa, rows);
+            else if (nkb <= 32 * 32) select_topk_kernel<32><<<grid, 256, tbl, stream>>>(sa, rows);
+            else select_topk_kernel<128><<<grid, 256, tbl, stream>>>(sa, rows);
         } else {
             // cumulative-mass mode needs the sorted order: shared-memory bitonic sort, one CTA per row
             size_t smem = size_t(sa.npad) * 8 * 2 + ((nkb + 15) & ~15);
