@@ -28,8 +28,9 @@ Pin status (tests/test_oracle_*.py):
   pooled_scores ..................... pinned (bilinearity identity vs. per-token brute force)
   forced_blocks ..................... pinned (per-token brute force)
   select_topk / select_cummass ...... pinned (stable sort, counts, order and minimality invariants)
+  block_mass_exact / select_by_mass / build_connectivity_exact ... pinned (brute force, closed form, invariants)
   fidelity of the pooled estimator to the true block attention mass: PARITY UNPINNED
-  (the paper prints no mask, density or recall figure; block_mass_exact only reports it).
+  (the paper prints no mask, density or recall figure; it can only be reported, see tests).
 """
 from __future__ import annotations
 
@@ -313,22 +314,69 @@ def build_connectivity(Qb, Kb, N, n_text, T, Hg, Wg, block_q, block_k, scale,
     return mask, scores, theta, F
 
 
-def block_mass_exact(Qb_head, Kb_head, N, block_q, block_k, scale) -> np.ndarray:
-    """The paper's literal quantity, for reporting only (tiny inputs): the share of a
-    query block's softmax attention mass that falls in each key block, averaged over
-    the block's queries.  [nqb, nkb] fp64, rows sum to 1."""
+def block_mass_exact(Qb_head, Kb_head, N, block_q, block_k, scale, lse: Optional[np.ndarray] = None) -> np.ndarray:
+    """The paper's literal quantity (Appendix "Reuse-Scope Implementation Details": the attention
+    mass a query block sends to each key block): mass[I, J] = (1/|I|) * sum_{i in I} sum_{j in J}
+    exp(s_ij - LSE_i), LSE_i the log-sum-exp of query i over ALL keys.  [nqb, nkb] fp64; each row
+    sums to 1.  ``lse`` (natural log, [N]) may be supplied -- e.g. the LSE a dense attention run
+    returned; otherwise it is computed here from the same scores."""
     q = _widen(Qb_head[:N])
     k = _widen(Kb_head[:N])
-    s = scale * (q @ k.T)
-    p = np.exp(s - s.max(axis=1, keepdims=True))
-    p /= p.sum(axis=1, keepdims=True)
     nqb, nkb = -(-N // block_q), -(-N // block_k)
+    starts = np.arange(nkb) * block_k
     out = np.zeros((nqb, nkb))
     for I in range(nqb):
-        rows = p[I * block_q: min(N, (I + 1) * block_q)]
-        for J in range(nkb):
-            out[I, J] = rows[:, J * block_k: min(N, (J + 1) * block_k)].sum() / rows.shape[0]
+        i0, i1 = I * block_q, min(N, (I + 1) * block_q)
+        s = scale * (q[i0:i1] @ k.T)
+        l = lse[i0:i1, None] if lse is not None else np.logaddexp.reduce(s, axis=1, keepdims=True)
+        p = np.exp(s - l)
+        out[I] = np.add.reduceat(p, starts, axis=1).sum(axis=0) / (i1 - i0)
     return out
+
+
+def select_by_mass(mass_row: np.ndarray, forced_row: np.ndarray, target: float):
+    """Smallest descending prefix of the non-forced key blocks whose mass, together with the forced
+    blocks', reaches ``target`` of the row's total (ties: lower block index first).  Returns
+    (keep bool[nkb], theta) with theta the mass of the last admitted block (NaN if none)."""
+    m = mass_row.astype(np.float64)
+    p = m / m.sum()
+    keep = forced_row.copy()
+    free = np.nonzero(~forced_row)[0]
+    ranked = _descending_stable(mass_row, free)
+    tgt = float(np.float32(target))
+    running = float(p[forced_row].sum())
+    theta = np.float32(np.nan)
+    for J in ranked:
+        if running >= tgt:
+            break
+        keep[J] = True
+        running += p[J]
+        theta = mass_row[J]
+    return keep, theta
+
+
+def build_connectivity_exact(Qb, Kb, N, n_text, T, Hg, Wg, block_q, block_k, scale, mass=0.9,
+                             window_frames=-1, text_dense=0, lse: Optional[np.ndarray] = None,
+                             heads: Optional[Iterable[Tuple[int, int]]] = None):
+    """The paper's rule on the exact block masses: per head and query block keep the smallest set of
+    key blocks covering ``mass`` of the attention mass (always-kept blocks included).  ``lse`` is
+    [B, H, N] or None.  Returns mask uint8, masses float32 [B,H,nqb,nkb], theta, forced table."""
+    B, H = Qb.shape[0], Qb.shape[1]
+    nqb, nkb = -(-N // block_q), -(-N // block_k)
+    F = forced_blocks(N, n_text, T, Hg, Wg, block_q, block_k, window_frames, text_dense)
+    mask = np.zeros((B, H, nqb, nkb), dtype=np.uint8)
+    masses = np.zeros((B, H, nqb, nkb), dtype=np.float32)
+    theta = np.full((B, H, nqb), np.nan, dtype=np.float32)
+    todo = list(heads) if heads is not None else [(b, h) for b in range(B) for h in range(H)]
+    for (b, h) in todo:
+        M = block_mass_exact(Qb[b, h], Kb[b, h], N, block_q, block_k, scale,
+                             None if lse is None else lse[b, h]).astype(np.float32)
+        masses[b, h] = M
+        for I in range(nqb):
+            keep, th = select_by_mass(M[I], F[I], mass)
+            mask[b, h, I] = keep
+            theta[b, h, I] = th
+    return mask, masses, theta, F
 
 
 # ==========================================================================

@@ -189,3 +189,97 @@ def test_block_mass_rows_sum_to_one_and_estimator_recall_reported():
     Q, K, _ = wl.gen_qkv(w)
     M = orc.block_mass_exact(Q[0, 0], K[0, 0], w.N, 64, 64, w.scale)
     np.testing.assert_allclose(M.sum(-1), 1.0, atol=1e-12)
+
+
+# ---------------------------------------------------------------------------------------------
+# exact block-mass rule (the paper's literal statement)
+# ---------------------------------------------------------------------------------------------
+def _mass_bruteforce(Q, K, N, bq, bk, scale):
+    q, k = widen(Q), widen(K)
+    nqb, nkb = -(-N // bq), -(-N // bk)
+    out = np.zeros((nqb, nkb))
+    for i in range(N):
+        s = [scale * sum(q[i, d] * k[j, d] for d in range(q.shape[1])) for j in range(N)]
+        mx = max(s)
+        den = sum(math.exp(v - mx) for v in s)
+        for j in range(N):
+            out[i // bq, j // bk] += math.exp(s[j] - mx) / den
+    for I in range(nqb):
+        out[I] /= min(bq, N - I * bq)
+    return out
+
+
+def test_block_mass_matches_bruteforce_and_rows_sum_to_one():
+    rng = np.random.default_rng(20)
+    N, D, bq, bk = 37, 4, 8, 16
+    Q, K = rand_bits(rng, (N, D)), rand_bits(rng, (N, D))
+    M = orc.block_mass_exact(Q, K, N, bq, bk, 0.7)
+    np.testing.assert_allclose(M, _mass_bruteforce(Q, K, N, bq, bk, 0.7), atol=1e-12)
+    np.testing.assert_allclose(M.sum(-1), 1.0, atol=1e-12)
+
+
+def test_block_mass_uniform_case_and_supplied_lse():
+    """Q = 0 => every key gets 1/N, so mass[I, J] = |J| / N exactly; an LSE taken from the (pinned)
+    attention oracle's dense run gives the same masses as the internal one."""
+    rng = np.random.default_rng(21)
+    N, D = 45, 8
+    Q, K, V = (rand_bits(rng, (1, 1, N, D)) for _ in range(3))
+    M0 = orc.block_mass_exact(np.zeros_like(Q[0, 0]), K[0, 0], N, 16, 8, 0.3)
+    sizes = np.minimum(8, N - np.arange(6) * 8) / N
+    np.testing.assert_allclose(M0, np.tile(sizes, (3, 1)), atol=1e-12)
+    ones = np.ones((1, 1, 3, 6), dtype=np.uint8)
+    _, L = orc.attention_full(Q, K, V, N, 16, 8, 0.3, ones)
+    np.testing.assert_allclose(orc.block_mass_exact(Q[0, 0], K[0, 0], N, 16, 8, 0.3, lse=L[0, 0]),
+                               orc.block_mass_exact(Q[0, 0], K[0, 0], N, 16, 8, 0.3), atol=1e-12)
+
+
+def test_select_by_mass_is_smallest_covering_descending_prefix():
+    rng = np.random.default_rng(22)
+    for trial in range(60):
+        n = int(rng.integers(2, 40))
+        m = rng.random(n).astype(np.float32) ** 4
+        m[rng.random(n) < 0.2] = m[0]                     # ties
+        forced = rng.random(n) < 0.15
+        tau = float(rng.choice([0.5, 0.9, 0.99]))
+        keep, theta = orc.select_by_mass(m, forced, tau)
+        p = m.astype(np.float64) / m.astype(np.float64).sum()
+        t32 = float(np.float32(tau))
+        assert keep[forced].all() and p[keep].sum() >= t32 - 1e-12
+        adm = keep & ~forced
+        if adm.any():
+            weakest = min(np.nonzero(adm)[0], key=lambda j: (float(m[j]), -j))
+            assert p[keep].sum() - p[weakest] < t32            # minimal
+            assert theta == m[weakest]
+            if (~keep).any():
+                assert m[adm].min() >= m[~keep].max()          # a descending prefix
+            # equal masses: lower index first
+            eq = [j for j in range(n) if not forced[j] and m[j] == m[weakest]]
+            kept_eq = [j for j in eq if keep[j]]
+            assert kept_eq == eq[:len(kept_eq)]
+        else:
+            assert p[forced].sum() >= t32
+
+
+def test_exact_rule_agrees_with_cummass_rule_on_log_masses():
+    """select_cummass on scores = ln(mass) is the same rule (softmax of ln m = m / sum m)."""
+    rng = np.random.default_rng(23)
+    m = (rng.random(24) ** 3 + 1e-3).astype(np.float32)
+    forced = np.zeros(24, dtype=bool); forced[3] = True
+    k1, _ = orc.select_by_mass(m, forced, 0.8)
+    k2, _ = orc.select_cummass(np.log(m.astype(np.float64)).astype(np.float32), forced, 0.8)
+    np.testing.assert_array_equal(k1, k2)
+
+
+def test_build_connectivity_exact_and_estimator_recall_is_reported():
+    """Exact rule on a structured slice; the recall of the pooled estimator against it is only reported."""
+    w = wl.shrunk(wl.get("wan1p3b_480p"), H=1, T=4, Hg=16, Wg=16)
+    Q, K, _ = wl.gen_qkv(w, "history")
+    mask, masses, theta, F = orc.build_connectivity_exact(Q, K, w.N, 0, w.T, w.Hg, w.Wg, 128, 128, w.scale, mass=0.9)
+    np.testing.assert_allclose(masses.sum(-1), 1.0, atol=1e-5)
+    kept = (masses * (mask != 0)).sum(-1)
+    assert (kept >= 0.9 - 1e-6).all()
+    est, _, _, _ = orc.build_connectivity(Q, K, w.N, 0, w.T, w.Hg, w.Wg, 128, 128, w.scale,
+                                          orc.MODE_CUMMASS, 0.25, 0.9, -1, 0, 1)
+    recall = float(((est != 0) & (mask != 0)).sum() / max(1, (mask != 0).sum()))
+    print(f"pooled estimator recall of the exact 0.9-mass blocks: {recall:.3f}")
+    assert 0.0 <= recall <= 1.0
