@@ -44,6 +44,8 @@ def parse_args():
     ap.add_argument("--density", type=float, default=None, help="override the builder's keep ratio")
     ap.add_argument("--attn-impl", default="auto", choices=["auto", "portable", "tcgen05"])
     ap.add_argument("--heads", type=int, default=None, help="run a slice with fewer heads (profiling captures)")
+    ap.add_argument("--exact-builder", action="store_true",
+                    help="also time carnator_build_connectivity_exact (block masses on the tensor cores) on the history pair")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -326,6 +328,34 @@ def run_ours(args):
     ms_step = total_ms / args.steps
     value = whole_job_tflops(flops, world, ms_step)
 
+    # ---- optional: the exact block-mass builder (second pass over Q K^T with the dense run's LSE) --------
+    exact = None
+    if args.exact_builder:
+        ones = torch.ones((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=dev)
+        Vz = torch.zeros_like(Kh)
+        hsh = cn.shape_of(w, Qh, Kh, Vz, None, attn_impl=impl)
+        _, Lh, _ = cn.sparse_attn(Qh, Kh, Vz, ones, None, hsh)
+        del Vz, ones
+        xparams = cn.params_of(dataclasses.replace(w.build, mode=wl.MODE_CUMMASS))
+        xmask = torch.empty((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=dev)
+        xws = torch.empty(cn.exact_workspace_bytes(bshape), dtype=torch.uint8, device=dev)
+        for _ in range(3):
+            cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, ws=xws)
+        torch.cuda.synchronize()
+        n_x = max(3, min(args.steps, 10))
+        xe = [torch.cuda.Event(enable_timing=True) for _ in range(n_x + 1)]
+        xe[0].record()
+        for i in range(n_x):
+            cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, ws=xws)
+            xe[i + 1].record()
+        torch.cuda.synchronize()
+        x_ms = float(np.mean([xe[i].elapsed_time(xe[i + 1]) for i in range(n_x)]))
+        x_flops = 2.0 * w.B * w.H * float(w.N) * float(w.N) * w.D
+        exact = {"ms": x_ms, "tflops": x_flops / (x_ms * 1e-3) / 1e12, "frac": x_flops / (x_ms * 1e-3) / 1e12 / peaks["bf16"],
+                 "flops_per_launch": x_flops, "mass": w.build.mass, "density": float(xmask.float().mean()),
+                 "status": cn.query_status(xws), "steps": n_x, "bound": "tensor", "peak": peaks["bf16"]}
+        del Lh, xmask, xws
+
     # ---- end to end through the host-buffer calls --------------------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -403,6 +433,8 @@ def run_ours(args):
         "attn_tflops": attn_tflops, "clocks": clocks, "gpu_launches": int(launches),
         "roofline": roofline, "builder_roofline": builder, "cpu_baseline": cpu, "e2e": e2e,
     }
+    if exact is not None:
+        line["exact_builder"] = exact
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

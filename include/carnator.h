@@ -115,6 +115,33 @@ carnator_status carnator_build_connectivity(const void* Q, const void* K,
                                             void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Connectivity builder on the exact block attention mass (cache-write side).
+ *
+ * Paper: Appendix "Reuse-Scope Implementation Details", stated literally -- per head and query
+ * block, the smallest set of key blocks covering a fixed fraction of the attention mass, where
+ *   mass[I,J] = (1/|I|) * sum_{i in I} sum_{j in J} exp(s_ij - LSE_i)
+ * is the share of query block I's softmax attention that falls into key block J (rows sum to 1).
+ * LSE is the log-sum-exp over all keys that a dense run of carnator_sparse_attn (all-ones mask)
+ * returns for the same Q and K, so this call is a second pass over Q K^T on the tensor cores
+ * followed by the cumulative-mass selection (ties: lower key-block index first; the always-kept
+ * blocks of `params` count towards the covered mass).
+ *
+ *   Q, K    device, bf16, strides of `shape`;  LSE  device, fp32 [B,H,N] contiguous, natural log
+ *   params  mass, window_frames and text_dense are used; mode / keep_ratio are ignored
+ *   mask    device, uint8 [B,H,nqb,nkb], written
+ *   block_mass_opt  device, fp32 [B,H,nqb,nkb] or NULL; receives the masses
+ *   ws      device workspace, 256-byte aligned, >= carnator_exact_workspace_bytes
+ * Limits: block_q = block_k = 128, nkb <= 4096.
+ * ------------------------------------------------------------------------ */
+size_t carnator_exact_workspace_bytes(const carnator_shape* shape);
+
+carnator_status carnator_build_connectivity_exact(const void* Q, const void* K, const float* LSE,
+                                                  const carnator_shape* shape,
+                                                  const carnator_build_params* params,
+                                                  uint8_t* mask, float* block_mass_opt,
+                                                  void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * Sparse attention under a reused mask (cache-hit side).
  *
  * Paper: Section 3.3, "Historical Sparse-Connectivity Reuse" (the target's Q, K,

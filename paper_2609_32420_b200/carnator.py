@@ -22,6 +22,7 @@ MODE_TOPK, MODE_CUMMASS = 0, 1
 # every symbol include/carnator.h declares
 EXPORTS = [
     "carnator_build_workspace_bytes", "carnator_build_connectivity",
+    "carnator_exact_workspace_bytes", "carnator_build_connectivity_exact",
     "carnator_attn_workspace_bytes", "carnator_compact_mask", "carnator_sparse_attn_compacted",
     "carnator_sparse_attn", "carnator_compacted_tiles",
     "carnator_attn_host_arena_bytes", "carnator_sparse_attn_host",
@@ -90,6 +91,10 @@ def lib() -> ctypes.CDLL:
     L.carnator_build_workspace_bytes.argtypes = [ps, pp]
     L.carnator_build_connectivity.restype = ctypes.c_int
     L.carnator_build_connectivity.argtypes = [vp, vp, ps, pp, vp, vp, vp, sz, vp]
+    L.carnator_exact_workspace_bytes.restype = sz
+    L.carnator_exact_workspace_bytes.argtypes = [ps]
+    L.carnator_build_connectivity_exact.restype = ctypes.c_int
+    L.carnator_build_connectivity_exact.argtypes = [vp, vp, vp, ps, pp, vp, vp, vp, sz, vp]
     L.carnator_attn_workspace_bytes.restype = sz
     L.carnator_attn_workspace_bytes.argtypes = [ps]
     L.carnator_compact_mask.restype = ctypes.c_int
@@ -215,6 +220,24 @@ def build_connectivity(Q, K, shape: Shape, params: BuildParams, mask=None, poole
     st = lib().carnator_build_connectivity(_ptr(Q), _ptr(K), ctypes.byref(shape), ctypes.byref(params), _ptr(mask),
                                            _ptr(pooled_scores), _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "carnator_build_connectivity")
+    return mask, ws
+
+
+def exact_workspace_bytes(shape: Shape) -> int:
+    return int(lib().carnator_exact_workspace_bytes(ctypes.byref(shape)))
+
+
+def build_connectivity_exact(Q, K, LSE, shape: Shape, params: BuildParams, mask=None, block_mass=None, ws=None,
+                             stream=None):
+    """carnator_build_connectivity_exact.  Returns (mask uint8 [B,H,nqb,nkb], ws)."""
+    import torch
+    if mask is None:
+        mask = torch.empty((shape.B, shape.H, shape.nqb, shape.nkb), dtype=torch.uint8, device=Q.device)
+    if ws is None:
+        ws = _new_ws(exact_workspace_bytes(shape), Q.device)
+    st = lib().carnator_build_connectivity_exact(_ptr(Q), _ptr(K), _ptr(LSE), ctypes.byref(shape), ctypes.byref(params),
+                                                 _ptr(mask), _ptr(block_mass), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "carnator_build_connectivity_exact")
     return mask, ws
 
 

@@ -188,6 +188,7 @@ struct SelectArgs {
     float keep_ratio, mass;
     int count_includes_forced;
     int k_all;             // top-k count over all nkb blocks (host computed)
+    int values_are_mass;   // cumulative-mass mode on non-negative block masses: p = value / sum instead of a softmax
     Geometry g;
 };
 
@@ -255,7 +256,7 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
         for (int w = 1; w < (nt >> 5); ++w) rmax = fmaxf(rmax, fscratch[w]);
         double my_all = 0.0, my_fm = 0.0;
         for (int J = tid; J < a.nkb; J += nt) {
-            double e = exp(double(s[J]) - double(rmax));
+            double e = a.values_are_mass ? double(s[J]) : exp(double(s[J]) - double(rmax));
             my_all += e;
             if (keep[J]) my_fm += e;
         }
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(256) select_kernel(SelectArgs a) {
             double p = 0.0;
             if (t < nfree) {
                 int J = int(0xFFFFFFFFu - uint32_t(keys[t] & 0xFFFFFFFFull));
-                p = exp(double(s[J]) - double(rmax)) / total;
+                p = (a.values_are_mass ? double(s[J]) : exp(double(s[J]) - double(rmax))) / total;
             }
             pm[t] = p;
         }

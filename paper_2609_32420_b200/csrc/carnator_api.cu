@@ -11,6 +11,7 @@
 #include "compact.cuh"
 #include "attn_portable.cuh"
 #include "attn_tcgen05.cuh"
+#include "block_mass_tcgen05.cuh"
 
 using namespace carnator;
 
@@ -171,6 +172,7 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
         sa.mode = p->mode; sa.keep_ratio = p->keep_ratio; sa.mass = p->mass;
         sa.count_includes_forced = p->count_includes_forced;
         sa.k_all = topk_count_host(p->keep_ratio, nkb);
+        sa.values_are_mass = 0;
         sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
         sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
         if (p->mode == CARNATOR_MODE_TOPK) {
@@ -192,6 +194,74 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
         }
         LAUNCH_CHECK("select_kernel");
     }
+    return CARNATOR_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// exact block-mass builder
+// ------------------------------------------------------------------------------------------------
+namespace {
+struct ExactWs { WsHeader* hdr; float* mass; size_t bytes; };
+ExactWs exact_ws_layout(void* base, int B, int H, int nqb, int nkb) {
+    ExactWs w;
+    char* p = static_cast<char*>(base);
+    w.hdr = reinterpret_cast<WsHeader*>(p);
+    w.mass = reinterpret_cast<float*>(p + align256(sizeof(WsHeader)));
+    w.bytes = align256(sizeof(WsHeader)) + align256(size_t(B) * H * nqb * size_t(nkb) * 4);
+    return w;
+}
+}  // namespace
+
+extern "C" size_t carnator_exact_workspace_bytes(const carnator_shape* s) {
+    if (check_shape(s, false) != CARNATOR_OK) return 0;
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    return exact_ws_layout(nullptr, s->B, s->H, nqb, nkb).bytes;
+}
+
+extern "C" carnator_status carnator_build_connectivity_exact(const void* Q, const void* K, const float* LSE,
+                                                             const carnator_shape* s, const carnator_build_params* p,
+                                                             uint8_t* mask, float* block_mass_opt, void* ws,
+                                                             size_t ws_bytes, void* stream_) {
+    carnator_status st = check_shape(s, false);
+    if (st != CARNATOR_OK) return st;
+    if (!p) return CARNATOR_ERR_INVALID_ARG;
+    if (!(p->mass > 0.f && p->mass <= 1.f) || p->window_frames < -1) return CARNATOR_ERR_INVALID_ARG;
+    if (!Q || !K || !LSE || !mask) return CARNATOR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(LSE, 4)) return CARNATOR_ERR_INVALID_ARG;
+    if (block_mass_opt && !aligned(block_mass_opt, 4)) return CARNATOR_ERR_INVALID_ARG;
+    if (s->block_q != tc::kBlock || s->block_k != tc::kBlock) return CARNATOR_ERR_UNSUPPORTED;
+    const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
+    if (nkb > kMaxKeyBlocksBuilder) return CARNATOR_ERR_UNSUPPORTED;
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    ExactWs w = exact_ws_layout(ws, s->B, s->H, nqb, nkb);
+    if (ws_bytes < w.bytes) return CARNATOR_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    float* mass = block_mass_opt ? block_mass_opt : w.mass;
+    CUDA_TRY(cudaMemsetAsync(w.hdr, 0, sizeof(WsHeader), stream));
+
+    tc::MassArgs ma;
+    ma.LSE = LSE; ma.mass = mass; ma.hdr = w.hdr;
+    ma.B = s->B; ma.H = s->H; ma.N = s->N; ma.nqb = nqb; ma.nkb = nkb;
+    ma.scale_log2 = effective_scale(s) * kLog2e;
+    st = launch_block_mass(Q, K, s->q_stride, s->k_stride, ma, s->D, stream, g_cuda_error, sizeof(g_cuda_error));
+    if (st != CARNATOR_OK) return st;
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+
+    SelectArgs sa;
+    sa.scores = mass; sa.mask = mask;
+    sa.nqb = nqb; sa.nkb = nkb; sa.npad = next_pow2(nkb); sa.H = s->H;
+    sa.mode = CARNATOR_MODE_CUMMASS; sa.keep_ratio = 1.f; sa.mass = p->mass;
+    sa.count_includes_forced = 1; sa.k_all = nkb; sa.values_are_mass = 1;
+    sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
+    sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
+    const size_t smem = size_t(sa.npad) * 8 * 2 + ((nkb + 15) & ~15);
+    st = allow_smem(select_kernel, 72 * 1024);
+    if (st != CARNATOR_OK) return st;
+    dim3 grid(nqb, s->H, s->B);
+    select_kernel<<<grid, 256, smem, stream>>>(sa);
+    LAUNCH_CHECK("select_kernel");
     return CARNATOR_OK;
 }
 
