@@ -29,6 +29,7 @@ Pin status (tests/test_oracle_*.py):
   forced_blocks ..................... pinned (per-token brute force)
   select_topk / select_cummass ...... pinned (stable sort, counts, order and minimality invariants)
   block_mass_exact / select_by_mass / build_connectivity_exact ... pinned (brute force, closed form, invariants)
+  build_regions / fuse_latents / region_block_flags / attention_region_rows ... pinned (definitions by hand, closed forms)
   fidelity of the pooled estimator to the true block attention mass: PARITY UNPINNED
   (the paper prints no mask, density or recall figure; it can only be reported, see tests).
 """
@@ -377,6 +378,91 @@ def build_connectivity_exact(Qb, Kb, N, n_text, T, Hg, Wg, block_q, block_k, sca
             mask[b, h, I] = keep
             theta[b, h, I] = th
     return mask, masses, theta, F
+
+
+# ==========================================================================
+# Reuse regions, latent fusion, region-restricted connectivity
+# (Section 3.3 "Region-Guided Latent Reuse" and "Joint Reuse in Intermediate Layers";
+#  Appendix "Reuse-Scope Implementation Details")
+# ==========================================================================
+def chebyshev_distance_per_frame(src: np.ndarray) -> np.ndarray:
+    """For every token of a [T, H, W] grid, the Chebyshev distance (max of row and column offsets)
+    to the nearest True token of ``src`` in the SAME frame; a large number (T*H*W) where the frame
+    holds none.  Plain search, written for small grids."""
+    T, H, W = src.shape
+    big = T * H * W
+    out = np.full((T, H, W), big, dtype=np.int64)
+    for t in range(T):
+        ys, xs = np.nonzero(src[t])
+        if len(ys) == 0:
+            continue
+        for y in range(H):
+            for x in range(W):
+                out[t, y, x] = np.maximum(np.abs(ys - y), np.abs(xs - x)).min()
+    return out
+
+
+def dilate_per_frame(src: np.ndarray, radius: int) -> np.ndarray:
+    """Dilation by ``radius`` tokens on the H x W grid of each latent frame (square neighbourhood,
+    i.e. every token within Chebyshev distance ``radius`` of the region; no wrap-around)."""
+    return chebyshev_distance_per_frame(src) <= radius
+
+
+def smoothstep(x):
+    return 3.0 * x * x - 2.0 * x * x * x
+
+
+def build_regions(evidence: np.ndarray, r_active: int = 2, r_context: int = 3):
+    """Active region = evidence dilated by r_active, context region = active dilated by a further
+    r_context (per latent frame).  Blend weight W: 1 on the evidence region, 1 - smoothstep(d_hat)
+    on the transition band active minus evidence, 0 outside the active region, where d_hat is the
+    Chebyshev distance to the evidence region divided by the largest such distance attained in the
+    band (taken over the whole band).  Returns (active bool, context bool, W float64), all [T, H, W]."""
+    ev = evidence != 0
+    d = chebyshev_distance_per_frame(ev)
+    active = d <= r_active
+    context = chebyshev_distance_per_frame(active) <= r_context
+    band = active & ~ev
+    W = np.zeros(ev.shape, dtype=np.float64)
+    W[ev] = 1.0
+    if band.any():
+        dmax = float(d[band].max())
+        W[band] = 1.0 - smoothstep(d[band] / dmax)
+    return active, context, W
+
+
+def fuse_latents(z_target: np.ndarray, z_hist: np.ndarray, W: np.ndarray) -> np.ndarray:
+    """z = W * z_target + (1 - W) * z_hist, W broadcast over the leading (channel) axes; fp64."""
+    zt = np.asarray(z_target, dtype=np.float64)
+    zh = np.asarray(z_hist, dtype=np.float64)
+    return W * zt + (1.0 - W) * zh
+
+
+def region_block_flags(region: np.ndarray, n_text: int, block: int, text_value: int = 1) -> np.ndarray:
+    """uint8 per block of the token order (text first, then the grid flattened frame-major): 1 if the
+    block holds a token of the region.  Text tokens count as members when text_value is 1."""
+    flat = np.concatenate([np.full(n_text, bool(text_value)), (region != 0).ravel()])
+    nb = -(-flat.size // block)
+    out = np.zeros(nb, dtype=np.uint8)
+    for I in range(nb):
+        out[I] = 1 if flat[I * block:(I + 1) * block].any() else 0
+    return out
+
+
+def attention_region_rows(Qb, Kb, Vb, N, block_q, block_k, scale, mask, active_q, context_k, rows):
+    """Middle-layer form: the historical connectivity restricted to active query blocks and context key
+    blocks (mask AND active x context); query blocks that are not active are not computed at all (their
+    rows come back NaN: the caller keeps the cached values).  active_q [B, nqb], context_k [B, nkb]."""
+    B = mask.shape[0]
+    eff = mask.copy()
+    for b in range(B):
+        eff[b] = mask[b] * (context_k[b] != 0)[None, None, :]
+    O, L = attention_rows(Qb, Kb, Vb, N, block_q, block_k, scale, eff, None, rows)
+    for r, (b, h, I) in enumerate(rows):
+        if active_q[b, I] == 0:
+            O[r] = np.nan
+            L[r] = np.nan
+    return O, L
 
 
 # ==========================================================================
