@@ -46,6 +46,8 @@ def parse_args():
     ap.add_argument("--heads", type=int, default=None, help="run a slice with fewer heads (profiling captures)")
     ap.add_argument("--exact-builder", action="store_true",
                     help="also time carnator_build_connectivity_exact (block masses on the tensor cores) on the history pair")
+    ap.add_argument("--regions", action="store_true",
+                    help="also time the region builder, latent fusion and the region-restricted attention form")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -356,6 +358,46 @@ def run_ours(args):
                  "status": cn.query_status(xws), "steps": n_x, "bound": "tensor", "peak": peaks["bf16"]}
         del Lh, xmask, xws
 
+    # ---- optional: reuse regions, latent fusion, region-restricted attention ---------------------------------
+    regions = None
+    if args.regions:
+        rng = np.random.default_rng(77)
+        ev = np.zeros((w.T, w.Hg, w.Wg), dtype=np.uint8)
+        cy, cx = w.Hg // 2, w.Wg // 2
+        for t in range(w.T):                                   # one drifting object tube, about 6 % of each frame
+            cy = int(np.clip(cy + rng.integers(-1, 2), 6, w.Hg - 7)); cx = int(np.clip(cx + rng.integers(-2, 3), 10, w.Wg - 11))
+            ev[t, cy - 5:cy + 6, cx - 9:cx + 10] = 1
+        evd = torch.from_numpy(ev).to(dev)
+
+        def timed(fn, n=20):
+            for _ in range(3):
+                fn()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(); e0.record()
+            for _ in range(n):
+                fn()
+            e1.record(); torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / n
+
+        ms_regions = timed(lambda: cn.build_regions(evd, shape, 2, 3))
+        act, ctx, Wt = cn.build_regions(evd, shape, 2, 3)
+        C_lat = 64                                             # latent channels per token (16 x 2 x 2 patch)
+        zt = torch.randn((C_lat, w.T * w.Hg * w.Wg), dtype=torch.float32, device=dev)
+        zh = torch.randn_like(zt); zo = torch.empty_like(zt)
+        ms_fuse = timed(lambda: cn.fuse_latents(zt, zh, Wt.reshape(-1), z_out=zo))
+        fuse_bytes = 3.0 * zt.numel() * 4 + Wt.numel() * 4
+        aq = cn.region_block_flags(act, shape, w.block, 1).reshape(1, -1).contiguous()
+        ck = cn.region_block_flags(ctx, shape, w.block, 1).reshape(1, -1).contiguous()
+        rws = torch.empty(cn.attn_workspace_bytes(shape), dtype=torch.uint8, device=dev)
+        ms_rattn = timed(lambda: cn.sparse_attn_region(Q, K, V, mask, aq, ck, shape, O, LSE, ws=rws), n=5)
+        rtiles = cn.compacted_tiles(shape, rws)
+        regions = {"ms_build_regions": ms_regions, "ms_fuse_latents": ms_fuse,
+                   "fuse_gbs": fuse_bytes / (ms_fuse * 1e-3) / 1e9, "fuse_frac_of_hbm": fuse_bytes / (ms_fuse * 1e-3) / 1e9 / peaks["hbm"],
+                   "active_query_blocks": int(aq.sum()), "context_key_blocks": int(ck.sum()),
+                   "ms_region_attn": ms_rattn, "region_tiles": rtiles,
+                   "region_attn_tflops": rtiles * 4.0 * w.block * w.block * w.D / (ms_rattn * 1e-3) / 1e12}
+        del zt, zh, zo, rws
+
     # ---- end to end through the host-buffer calls --------------------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -435,6 +477,8 @@ def run_ours(args):
     }
     if exact is not None:
         line["exact_builder"] = exact
+    if regions is not None:
+        line["regions"] = regions
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

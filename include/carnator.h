@@ -218,6 +218,54 @@ carnator_status carnator_build_connectivity_host(const void* Q, const void* K,
                                                  void* arena, size_t arena_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Reuse regions, latent fusion and the region-restricted (middle-layer) attention form.
+ *
+ * Paper: Section 3.3 "Region-Guided Latent Reuse" (evidence region inside active region inside context
+ * region; z = W*z_target + (1-W)*z_hist with W = 1 on the evidence region, 1 - smoothstep(d_hat) on the
+ * transition band, 0 outside the active region) and "Joint Reuse in Intermediate Layers" (historical
+ * connectivity kept only for active queries and their context tokens; tokens outside the active region
+ * keep their cached computation); Appendix "Reuse-Scope Implementation Details" (dilation by 2 tokens,
+ * then by a further 3, per latent frame on the H x W grid; Chebyshev distance to the evidence region
+ * normalised by the largest distance attained in the band).
+ *
+ * carnator_build_regions:  evidence uint8 [T,Hg,Wg] (non-zero = member) -> active, context uint8 [T,Hg,Wg]
+ *   and W fp32 [T,Hg,Wg]; r_active >= 1, r_context >= 0, r_active + r_context <= 32; the grid comes from
+ *   `shape` (only T, Hg, Wg are read).  ws >= carnator_regions_workspace_bytes, 256-byte aligned.
+ * carnator_fuse_latents:   z_out = W*z_target + (1-W)*z_hist over [channels, tokens] row-major tensors of
+ *   `dtype` (CARNATOR_DTYPE_*), W fp32 [tokens]; tokens must be a multiple of 16 bytes worth of elements;
+ *   z_out may alias z_target or z_hist.
+ * carnator_region_block_flags: flags[i] = 1 iff block i of the token order (text first, then the grid,
+ *   `block` tokens per block) holds a region token; text tokens count as members iff text_value != 0.
+ * carnator_sparse_attn_region: as carnator_sparse_attn, with the evaluated pairs restricted to
+ *   mask[b,h,I,J] != 0 && active_q[b,I] != 0 && context_k[b,J] != 0; query blocks with active_q == 0 are
+ *   skipped: their rows of O and LSE are left untouched (the caller keeps the cached values there).
+ *   active_q uint8 [B,nqb], context_k uint8 [B,nkb], both required.
+ * All pointers are device pointers.
+ * ------------------------------------------------------------------------ */
+enum { CARNATOR_DTYPE_F32 = 0, CARNATOR_DTYPE_BF16 = 1 };
+
+size_t carnator_regions_workspace_bytes(const carnator_shape* shape);
+
+carnator_status carnator_build_regions(const uint8_t* evidence, const carnator_shape* shape,
+                                       int32_t r_active, int32_t r_context,
+                                       uint8_t* active, uint8_t* context, float* W,
+                                       void* ws, size_t ws_bytes, void* stream);
+
+carnator_status carnator_fuse_latents(const void* z_target, const void* z_hist, const float* W,
+                                      int64_t channels, int64_t tokens, int32_t dtype,
+                                      void* z_out, void* stream);
+
+carnator_status carnator_region_block_flags(const uint8_t* region, const carnator_shape* shape,
+                                            int32_t block, int32_t text_value,
+                                            uint8_t* flags, void* stream);
+
+carnator_status carnator_sparse_attn_region(const void* Q, const void* K, const void* V,
+                                            const uint8_t* mask, const uint8_t* active_q, const uint8_t* context_k,
+                                            const carnator_shape* shape,
+                                            void* O, float* LSE,
+                                            void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * carnator_sparse_attn_static -- carnator_sparse_attn for callers that cannot provide a workspace.
  *
  * (The paper has no counterpart for this call; it exists for deployment reasons only.)

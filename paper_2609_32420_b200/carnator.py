@@ -28,6 +28,8 @@ EXPORTS = [
     "carnator_attn_host_arena_bytes", "carnator_sparse_attn_host",
     "carnator_build_host_arena_bytes", "carnator_build_connectivity_host",
     "carnator_sparse_attn_static",
+    "carnator_regions_workspace_bytes", "carnator_build_regions", "carnator_fuse_latents",
+    "carnator_region_block_flags", "carnator_sparse_attn_region",
     "carnator_query_status", "carnator_status_string", "carnator_last_cuda_error",
     "carnator_kernel_launches", "carnator_version",
 ]
@@ -115,6 +117,16 @@ def lib() -> ctypes.CDLL:
     L.carnator_build_connectivity_host.argtypes = [vp, vp, ps, pp, vp, vp, sz, vp]
     L.carnator_sparse_attn_static.restype = ctypes.c_int
     L.carnator_sparse_attn_static.argtypes = [vp, vp, vp, vp, vp, ps, vp, vp, vp]
+    L.carnator_regions_workspace_bytes.restype = sz
+    L.carnator_regions_workspace_bytes.argtypes = [ps]
+    L.carnator_build_regions.restype = ctypes.c_int
+    L.carnator_build_regions.argtypes = [vp, ps, ctypes.c_int32, ctypes.c_int32, vp, vp, vp, vp, sz, vp]
+    L.carnator_fuse_latents.restype = ctypes.c_int
+    L.carnator_fuse_latents.argtypes = [vp, vp, vp, i64, i64, ctypes.c_int32, vp, vp]
+    L.carnator_region_block_flags.restype = ctypes.c_int
+    L.carnator_region_block_flags.argtypes = [vp, ps, ctypes.c_int32, ctypes.c_int32, vp, vp]
+    L.carnator_sparse_attn_region.restype = ctypes.c_int
+    L.carnator_sparse_attn_region.argtypes = [vp, vp, vp, vp, vp, vp, ps, vp, vp, vp, sz, vp]
     L.carnator_query_status.restype = ctypes.c_int
     L.carnator_query_status.argtypes = [vp, vp]
     L.carnator_status_string.restype = ctypes.c_char_p
@@ -327,3 +339,51 @@ def sparse_attn_static(Q, K, V, mask, recompute_rows, shape: Shape, O, LSE, stre
     st = lib().carnator_sparse_attn_static(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), _ptr(recompute_rows),
                                            ctypes.byref(shape), _ptr(O), _ptr(LSE), _stream(stream))
     _check(st, "carnator_sparse_attn_static")
+
+
+DTYPE_F32, DTYPE_BF16 = 0, 1
+
+
+def build_regions(evidence, shape: Shape, r_active: int = 2, r_context: int = 3, stream=None):
+    """carnator_build_regions.  evidence uint8 [T,Hg,Wg] on the device -> (active, context, W)."""
+    import torch
+    active = torch.empty_like(evidence)
+    context = torch.empty_like(evidence)
+    W = torch.empty(evidence.shape, dtype=torch.float32, device=evidence.device)
+    ws = _new_ws(int(lib().carnator_regions_workspace_bytes(ctypes.byref(shape))), evidence.device)
+    st = lib().carnator_build_regions(_ptr(evidence), ctypes.byref(shape), r_active, r_context, _ptr(active), _ptr(context),
+                                      _ptr(W), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "carnator_build_regions")
+    return active, context, W
+
+
+def fuse_latents(z_target, z_hist, W, z_out=None, stream=None):
+    """carnator_fuse_latents over [channels, tokens] tensors (fp32 or bf16), W fp32 [tokens]."""
+    import torch
+    if z_out is None:
+        z_out = torch.empty_like(z_target)
+    dtype = DTYPE_F32 if z_target.dtype == torch.float32 else DTYPE_BF16
+    channels, tokens = z_target.shape[0], z_target[0].numel()
+    st = lib().carnator_fuse_latents(_ptr(z_target), _ptr(z_hist), _ptr(W), channels, tokens, dtype, _ptr(z_out), _stream(stream))
+    _check(st, "carnator_fuse_latents")
+    return z_out
+
+
+def region_block_flags(region, shape: Shape, block: int, text_value: int = 1, stream=None):
+    import torch
+    n = shape.n_text + shape.T * shape.Hg * shape.Wg
+    flags = torch.empty((-(-n // block),), dtype=torch.uint8, device=region.device)
+    st = lib().carnator_region_block_flags(_ptr(region), ctypes.byref(shape), block, text_value, _ptr(flags), _stream(stream))
+    _check(st, "carnator_region_block_flags")
+    return flags
+
+
+def sparse_attn_region(Q, K, V, mask, active_q, context_k, shape: Shape, O, LSE, ws=None, stream=None):
+    """carnator_sparse_attn_region: O and LSE are updated in place; rows of inactive query blocks stay as they are."""
+    if ws is None:
+        ws = _new_ws(attn_workspace_bytes(shape), Q.device)
+    shape.o_stride = (ctypes.c_int64 * 3)(*O.stride()[:3])
+    st = lib().carnator_sparse_attn_region(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), _ptr(active_q), _ptr(context_k),
+                                           ctypes.byref(shape), _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "carnator_sparse_attn_region")
+    return ws

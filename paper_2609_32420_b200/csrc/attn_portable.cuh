@@ -71,6 +71,7 @@ __global__ void __launch_bounds__(BQ * 2) attn_portable_kernel(AttnArgs a) {
     const int64_t bh = int64_t(b) * a.H + h;
     const int I = a.order[bh * a.nqb + blockIdx.x];
     const int count = a.counts[bh * a.nqb + I];
+    if (count < 0) return;                         // skipped query block (region-restricted form): output untouched
     const int32_t* list = a.lists + (bh * a.nqb + I) * int64_t(a.nkb);
     const int q0 = I * BQ;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;

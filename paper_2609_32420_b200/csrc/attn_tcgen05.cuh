@@ -212,6 +212,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     const int32_t* list = a.lists + (bh * a.nqb + I) * int64_t(a.nkb);
     const int q0 = I * kBlock;
 
+    if (T < 0) return;                      // skipped query block (region-restricted form): output untouched
     if (T == 0) {                           // nothing to attend to: O = 0, LSE = -inf
         if (tid < kBlock && q0 + tid < a.N) {
             __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(q0 + tid) * a.os[2];

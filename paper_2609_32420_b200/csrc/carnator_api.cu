@@ -12,6 +12,7 @@
 #include "attn_portable.cuh"
 #include "attn_tcgen05.cuh"
 #include "block_mass_tcgen05.cuh"
+#include "regions.cuh"
 
 using namespace carnator;
 
@@ -282,8 +283,9 @@ static carnator_status attn_ws_check(const carnator_shape* s, void* ws, size_t w
     return CARNATOR_OK;
 }
 
-extern "C" carnator_status carnator_compact_mask(const uint8_t* mask, const uint8_t* recompute_rows,
-                                                 const carnator_shape* s, void* ws, size_t ws_bytes, void* stream_) {
+static carnator_status compact_impl(const uint8_t* mask, const uint8_t* recompute_rows, const uint8_t* active_q,
+                                    const uint8_t* context_k, const carnator_shape* s, void* ws, size_t ws_bytes,
+                                    void* stream_) {
     carnator_status st = check_shape(s, true);
     if (st != CARNATOR_OK) return st;
     if (!mask) return CARNATOR_ERR_INVALID_ARG;
@@ -297,11 +299,17 @@ extern "C" carnator_status carnator_compact_mask(const uint8_t* mask, const uint
     if (nqb > 12000) return CARNATOR_ERR_UNSUPPORTED;   // order kernel keeps one head's counts in shared memory
     CUDA_TRY(cudaMemsetAsync(w.hdr, 0, sizeof(WsHeader), stream));
     const int rows = s->B * s->H * nqb;
-    compact_rows_kernel<<<ceil_div(rows, 8), 256, 0, stream>>>(mask, recompute_rows, s->B, s->H, nqb, nkb, w.counts, w.lists);
+    compact_rows_kernel<<<ceil_div(rows, 8), 256, 0, stream>>>(mask, recompute_rows, s->B, s->H, nqb, nkb, w.counts, w.lists,
+                                                               active_q, context_k);
     LAUNCH_CHECK("compact_rows_kernel");
     order_rows_kernel<<<s->B * s->H, 256, size_t(nqb) * 4, stream>>>(w.counts, nqb, w.order, w.hdr);
     LAUNCH_CHECK("order_rows_kernel");
     return CARNATOR_OK;
+}
+
+extern "C" carnator_status carnator_compact_mask(const uint8_t* mask, const uint8_t* recompute_rows,
+                                                 const carnator_shape* s, void* ws, size_t ws_bytes, void* stream_) {
+    return compact_impl(mask, recompute_rows, nullptr, nullptr, s, ws, ws_bytes, stream_);
 }
 
 template <int D, int BQ>
@@ -506,6 +514,89 @@ extern "C" carnator_status carnator_build_connectivity_host(const void* Q, const
     CUDA_TRY(cudaMemcpyAsync(mask, dM, mbytes, cudaMemcpyDeviceToHost, stream));
     CUDA_TRY(cudaStreamSynchronize(stream));
     return carnator_query_status(ws, stream_);
+}
+
+// ------------------------------------------------------------------------------------------------
+// reuse regions, latent fusion, region-restricted attention
+// ------------------------------------------------------------------------------------------------
+extern "C" size_t carnator_regions_workspace_bytes(const carnator_shape* s) {
+    if (!s || s->T <= 0 || s->Hg <= 0 || s->Wg <= 0) return 0;
+    return align256(sizeof(WsHeader)) + align256(size_t(s->T) * s->Hg * s->Wg);
+}
+
+extern "C" carnator_status carnator_build_regions(const uint8_t* evidence, const carnator_shape* s, int32_t r_active,
+                                                  int32_t r_context, uint8_t* active, uint8_t* context, float* W,
+                                                  void* ws, size_t ws_bytes, void* stream_) {
+    if (!s || s->T <= 0 || s->Hg <= 0 || s->Wg <= 0) return CARNATOR_ERR_INVALID_ARG;
+    if (!evidence || !active || !context || !W) return CARNATOR_ERR_INVALID_ARG;
+    if (r_active < 1 || r_context < 0 || r_active + r_context > 32) return CARNATOR_ERR_INVALID_ARG;
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    if (ws_bytes < carnator_regions_workspace_bytes(s)) return CARNATOR_ERR_WORKSPACE;
+    carnator_status st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    WsHeader* hdr = static_cast<WsHeader*>(ws);
+    uint8_t* dist = static_cast<uint8_t*>(ws) + align256(sizeof(WsHeader));
+    const int n = s->T * s->Hg * s->Wg;
+    CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WsHeader), stream));
+    region_distance_kernel<<<ceil_div(n, 256), 256, 0, stream>>>(evidence, s->T, s->Hg, s->Wg, r_active, r_context, dist,
+                                                                 active, context, hdr);
+    LAUNCH_CHECK("region_distance_kernel");
+    region_weight_kernel<<<ceil_div(n, 256), 256, 0, stream>>>(dist, n, r_active, hdr, W);
+    LAUNCH_CHECK("region_weight_kernel");
+    return CARNATOR_OK;
+}
+
+extern "C" carnator_status carnator_fuse_latents(const void* z_target, const void* z_hist, const float* W,
+                                                 int64_t channels, int64_t tokens, int32_t dtype, void* z_out,
+                                                 void* stream_) {
+    if (!z_target || !z_hist || !W || !z_out || channels <= 0 || tokens <= 0) return CARNATOR_ERR_INVALID_ARG;
+    if (dtype != CARNATOR_DTYPE_F32 && dtype != CARNATOR_DTYPE_BF16) return CARNATOR_ERR_INVALID_ARG;
+    const int vec = dtype == CARNATOR_DTYPE_F32 ? 4 : 8;
+    if (tokens % vec != 0) return CARNATOR_ERR_UNSUPPORTED;          // rows of 16 bytes
+    if (!aligned(z_target, 16) || !aligned(z_hist, 16) || !aligned(z_out, 16) || !aligned(W, 4)) return CARNATOR_ERR_INVALID_ARG;
+    carnator_status st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int64_t work = channels * (tokens / vec);
+    const unsigned grid = unsigned((work + 255) / 256);
+    if (dtype == CARNATOR_DTYPE_F32)
+        fuse_latents_kernel<float, 4><<<grid, 256, 0, stream>>>(static_cast<const float*>(z_target), static_cast<const float*>(z_hist),
+                                                               W, channels, tokens, static_cast<float*>(z_out));
+    else
+        fuse_latents_kernel<__nv_bfloat16, 8><<<grid, 256, 0, stream>>>(static_cast<const __nv_bfloat16*>(z_target),
+                                                                       static_cast<const __nv_bfloat16*>(z_hist), W, channels,
+                                                                       tokens, static_cast<__nv_bfloat16*>(z_out));
+    LAUNCH_CHECK("fuse_latents_kernel");
+    return CARNATOR_OK;
+}
+
+extern "C" carnator_status carnator_region_block_flags(const uint8_t* region, const carnator_shape* s, int32_t block,
+                                                       int32_t text_value, uint8_t* flags, void* stream_) {
+    if (!s || !region || !flags || block <= 0) return CARNATOR_ERR_INVALID_ARG;
+    if (s->n_text < 0 || s->T <= 0 || s->Hg <= 0 || s->Wg <= 0) return CARNATOR_ERR_INVALID_ARG;
+    carnator_status st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    const int n_video = s->T * s->Hg * s->Wg;
+    const int nblocks = ceil_div(s->n_text + n_video, block);
+    region_block_flags_kernel<<<ceil_div(nblocks, 8), 256, 0, stream>>>(region, s->n_text, n_video, block, text_value, nblocks, flags);
+    LAUNCH_CHECK("region_block_flags_kernel");
+    return CARNATOR_OK;
+}
+
+extern "C" carnator_status carnator_sparse_attn_region(const void* Q, const void* K, const void* V, const uint8_t* mask,
+                                                       const uint8_t* active_q, const uint8_t* context_k,
+                                                       const carnator_shape* s, void* O, float* LSE, void* ws,
+                                                       size_t ws_bytes, void* stream) {
+    carnator_status st = check_shape(s, true);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !V || !O || !LSE || !mask || !active_q || !context_k) return CARNATOR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(V, 16) || !aligned(O, 16) || !aligned(LSE, 4)) return CARNATOR_ERR_INVALID_ARG;
+    if (s->attn_impl == CARNATOR_IMPL_TCGEN05 && !tcgen05_supported(s)) return CARNATOR_ERR_UNSUPPORTED;
+    st = compact_impl(mask, nullptr, active_q, context_k, s, ws, ws_bytes, stream);
+    if (st != CARNATOR_OK) return st;
+    return carnator_sparse_attn_compacted(Q, K, V, s, O, LSE, ws, ws_bytes, stream);
 }
 
 // ------------------------------------------------------------------------------------------------
