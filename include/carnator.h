@@ -305,7 +305,14 @@ carnator_status carnator_sparse_attn_static(const void* Q, const void* K, const 
  * Status and diagnostics.
  * carnator_query_status synchronises `stream` and returns the status word that
  * kernels of earlier calls on this workspace may have set (CARNATOR_OK,
- * CARNATOR_ERR_DEVICE_TIMEOUT or CARNATOR_ERR_DEVICE_CHECK), then clears it.
+ * CARNATOR_ERR_DEVICE_TIMEOUT or CARNATOR_ERR_DEVICE_CHECK), then clears it.  The
+ * word is initialised by the calls that take the workspace (build, compact, the
+ * combined attention calls); querying a workspace no such call has used yet
+ * returns whatever the memory held.  CARNATOR_ERR_DEVICE_CHECK is raised by the
+ * tcgen05 attention kernel when a compacted list holds a key-block index outside
+ * [0, nkb) or is not strictly ascending (only possible if the workspace was
+ * modified between compaction and attention); the kernel then stops that query
+ * block before loading anything.
  * carnator_kernel_launches returns how many kernels this library has launched in
  * the calling process so far (monotone counter).
  * ------------------------------------------------------------------------ */

@@ -283,8 +283,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 if (!mbar_wait(bar_kempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
                 }
+                const int J = list[i];
+                if (J < 0 || J >= a.nkb || (i > 0 && J <= list[i - 1])) {      // malformed list: stop before touching memory
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_CHECK, 21, i, blockIdx.x); *abortp = 1; break;
+                }
                 mbar_expect_tx(bar_kfull(s), C::kTileBytes);
-                const int key0 = list[i] * kBlock;
+                const int key0 = J * kBlock;
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
                     tma_load_4d(sK + s * C::kTileBytes + x * C::kBoxBytes, &mapK, bar_kfull(s), x * 64, key0, h, b);
@@ -305,8 +309,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 if (!mbar_wait(bar_vempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
                 }
+                const int J = list[i];
+                if (J < 0 || J >= a.nkb) { *abortp = 1; break; }                  // reported by the K producer
                 mbar_expect_tx(bar_vfull(s), C::kTileBytes);
-                const int key0 = list[i] * kBlock;
+                const int key0 = J * kBlock;
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
                     tma_load_4d(sV + s * C::kTileBytes + x * C::kBoxBytes, &mapV, bar_vfull(s), x * 64, key0, h, b);

@@ -172,3 +172,29 @@ def test_full_size_workload_sampled_rows(name, density):
         assert bool((mask_dev == 1).all())
     # properties that hold at any size: every valid row finite, no row past N touched is checked above by shape
     assert torch.isfinite(O.float()).all() and torch.isfinite(L).all()
+
+
+def test_malformed_lists_are_reported_and_the_context_stays_usable():
+    """Host-made fault: the compacted lists are overwritten between compaction and attention.  The tcgen05 kernel
+    must stop the affected query block, report CARNATOR_ERR_DEVICE_CHECK, and leave the device usable."""
+    rng = np.random.default_rng(21)
+    B, H, N, D = 1, 1, 512, 128
+    Qb, Kb, Vb = (rand_bits(rng, (B, H, N, D)) for _ in range(3))
+    Q, K, V = to_dev(Qb), to_dev(Kb), to_dev(Vb)
+    shape = cn.make_shape(B, H, N, D, 0, 1, 1, N, 128, 128, Q, K, V, None, attn_impl=cn.IMPL_TCGEN05)
+    mask = torch.ones((B, H, 4, 4), dtype=torch.uint8, device="cuda")
+    ws = cn.compact_mask(mask, None, shape)
+    al = lambda x: (x + 255) // 256 * 256
+    lists_off = 256 + 2 * al(4 * 4)                     # header | counts | order | lists
+    lists = ws[lists_off: lists_off + 4 * 4 * 4].view(torch.int32)
+    assert lists[:4].tolist() == [0, 1, 2, 3]
+    lists[1] = 1_000_000                                # row 0 now points far outside the key blocks
+    O, L = cn.sparse_attn_compacted(Q, K, V, shape, ws)
+    assert cn.query_status(ws) == cn.ERR_DEVICE_CHECK
+    assert cn.query_status(ws) == cn.OK                 # reading the status clears it
+    # the same buffers, recompacted, run normally afterwards
+    ws = cn.compact_mask(mask, None, shape, ws=ws)
+    O, L = cn.sparse_attn_compacted(Q, K, V, shape, ws)
+    assert cn.query_status(ws) == cn.OK
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, N, 128, 128, 1.0 / np.sqrt(D), mask.cpu().numpy(), None)
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "after a reported list fault")
