@@ -266,6 +266,30 @@ carnator_status carnator_sparse_attn_region(const void* Q, const void* K, const 
                                             void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Host-side scalars of the reuse-validity gate and of its offline risk certificate.  No GPU work; all
+ * pointers are HOST pointers; invalid arguments give NaN (0 for the gate).
+ *
+ * Paper: Section 3.2 -- d_size = |log(A_q / A_j)|, d_shape = 1 - Dice of the bounding-box-normalised object
+ * indicators, d_context / d_color = CIEDE2000 difference of mean CIELAB colours, gate
+ * g_tau = prod_k 1[d_k <= tau_k] over the applicable dimensions; Appendix "Risk-Aware Compatibility
+ * Decision" -- one-sided Clopper-Pearson upper bound U_alpha(u, n) on the unsafe-reuse rate.
+ *
+ *   carnator_delta_e00            lab_a, lab_b: 3 doubles each (L*, a*, b*); k_L = k_C = k_H = 1
+ *   carnator_size_discrepancy     positive tail-slice areas
+ *   carnator_shape_discrepancy    binary indicators m_q [hq,wq], m_j [hj,wj]: each is cropped to its tight
+ *                                 support box and resampled (cell centres, nearest) to resolution x resolution
+ *   carnator_compatibility_gate   n dimensions; applicable may be NULL (= all); returns 1 iff all pass
+ *   carnator_clopper_pearson_upper  unsafe u of accepted n at one-sided level alpha: the p solving
+ *                                 P[Bin(n, p) <= u] = alpha (1 when u = n)
+ * ------------------------------------------------------------------------ */
+double  carnator_delta_e00(const double* lab_a, const double* lab_b);
+double  carnator_size_discrepancy(double area_q, double area_j);
+double  carnator_shape_discrepancy(const uint8_t* m_q, int32_t hq, int32_t wq,
+                                   const uint8_t* m_j, int32_t hj, int32_t wj, int32_t resolution);
+int32_t carnator_compatibility_gate(const double* d, const double* tau, const uint8_t* applicable, int32_t n);
+double  carnator_clopper_pearson_upper(int32_t unsafe, int32_t accepted, double alpha);
+
+/* ------------------------------------------------------------------------
  * carnator_sparse_attn_static -- carnator_sparse_attn for callers that cannot provide a workspace.
  *
  * (The paper has no counterpart for this call; it exists for deployment reasons only.)

@@ -30,6 +30,7 @@ Pin status (tests/test_oracle_*.py):
   select_topk / select_cummass ...... pinned (stable sort, counts, order and minimality invariants)
   block_mass_exact / select_by_mass / build_connectivity_exact ... pinned (brute force, closed form, invariants)
   build_regions / fuse_latents / region_block_flags / attention_region_rows ... pinned (definitions by hand, closed forms)
+  clopper_pearson_upper ... pinned (value printed in the paper, closed form for u = 0); delta_e00 / shape / size ... pinned (closed forms, invariants)
   fidelity of the pooled estimator to the true block attention mass: PARITY UNPINNED
   (the paper prints no mask, density or recall figure; it can only be reported, see tests).
 """
@@ -463,6 +464,75 @@ def attention_region_rows(Qb, Kb, Vb, N, block_q, block_k, scale, mask, active_q
             O[r] = np.nan
             L[r] = np.nan
     return O, L
+
+
+# ==========================================================================
+# Compatibility scalars and the risk certificate
+# (Section 3.2; Appendix "Risk-Aware Compatibility Decision")
+# ==========================================================================
+def delta_e00(lab1, lab2) -> float:
+    """CIEDE2000 colour difference (k_L = k_C = k_H = 1), vectorised-formula form in numpy."""
+    L1, a1, b1 = (float(v) for v in lab1)
+    L2, a2, b2 = (float(v) for v in lab2)
+    C1, C2 = np.hypot(a1, b1), np.hypot(a2, b2)
+    Cbar = (C1 + C2) / 2
+    G = 0.5 * (1 - np.sqrt(Cbar ** 7 / (Cbar ** 7 + 25.0 ** 7)))
+    a1p, a2p = (1 + G) * a1, (1 + G) * a2
+    C1p, C2p = np.hypot(a1p, b1), np.hypot(a2p, b2)
+    h1p = np.degrees(np.arctan2(b1, a1p)) % 360 if (a1p or b1) else 0.0
+    h2p = np.degrees(np.arctan2(b2, a2p)) % 360 if (a2p or b2) else 0.0
+    dLp, dCp = L2 - L1, C2p - C1p
+    if C1p * C2p == 0:
+        dhp = 0.0
+    else:
+        dhp = h2p - h1p
+        dhp = dhp - 360 if dhp > 180 else (dhp + 360 if dhp < -180 else dhp)
+    dHp = 2 * np.sqrt(C1p * C2p) * np.sin(np.radians(dhp / 2))
+    Lbar, Cbarp = (L1 + L2) / 2, (C1p + C2p) / 2
+    if C1p * C2p == 0:
+        hbar = h1p + h2p
+    elif abs(h1p - h2p) <= 180:
+        hbar = (h1p + h2p) / 2
+    else:
+        hbar = (h1p + h2p + 360) / 2 if h1p + h2p < 360 else (h1p + h2p - 360) / 2
+    T = (1 - 0.17 * np.cos(np.radians(hbar - 30)) + 0.24 * np.cos(np.radians(2 * hbar))
+         + 0.32 * np.cos(np.radians(3 * hbar + 6)) - 0.20 * np.cos(np.radians(4 * hbar - 63)))
+    dtheta = 30 * np.exp(-(((hbar - 275) / 25) ** 2))
+    RC = 2 * np.sqrt(Cbarp ** 7 / (Cbarp ** 7 + 25.0 ** 7))
+    SL = 1 + 0.015 * (Lbar - 50) ** 2 / np.sqrt(20 + (Lbar - 50) ** 2)
+    SC, SH = 1 + 0.045 * Cbarp, 1 + 0.015 * Cbarp * T
+    RT = -np.sin(np.radians(2 * dtheta)) * RC
+    return float(np.sqrt((dLp / SL) ** 2 + (dCp / SC) ** 2 + (dHp / SH) ** 2 + RT * (dCp / SC) * (dHp / SH)))
+
+
+def bbox_normalized(m: np.ndarray, res: int) -> np.ndarray:
+    """Crop a binary indicator to its tight support box and resample to res x res (nearest, cell centres)."""
+    ys, xs = np.nonzero(m)
+    box = m[ys.min():ys.max() + 1, xs.min():xs.max() + 1]
+    r = np.minimum(box.shape[0] - 1, ((np.arange(res) + 0.5) * box.shape[0] / res).astype(int))
+    c = np.minimum(box.shape[1] - 1, ((np.arange(res) + 0.5) * box.shape[1] / res).astype(int))
+    return (box[np.ix_(r, c)] != 0)
+
+
+def shape_discrepancy(m_q: np.ndarray, m_j: np.ndarray, res: int = 32) -> float:
+    a, b = bbox_normalized(m_q, res), bbox_normalized(m_j, res)
+    return 1.0 - 2.0 * float((a & b).sum()) / float(a.sum() + b.sum())
+
+
+def size_discrepancy(area_q: float, area_j: float) -> float:
+    return abs(math.log(area_q / area_j))
+
+
+def compatibility_gate(d, tau, applicable=None) -> int:
+    return int(all((dk <= tk) for k, (dk, tk) in enumerate(zip(d, tau)) if applicable is None or applicable[k]))
+
+
+def clopper_pearson_upper(u: int, n: int, alpha: float) -> float:
+    """One-sided upper limit: the (1 - alpha) quantile of Beta(u + 1, n - u) (library routine)."""
+    from scipy.stats import beta
+    if u >= n:
+        return 1.0
+    return float(beta.ppf(1.0 - alpha, u + 1, n - u))
 
 
 # ==========================================================================

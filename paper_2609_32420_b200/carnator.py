@@ -30,6 +30,8 @@ EXPORTS = [
     "carnator_sparse_attn_static",
     "carnator_regions_workspace_bytes", "carnator_build_regions", "carnator_fuse_latents",
     "carnator_region_block_flags", "carnator_sparse_attn_region",
+    "carnator_delta_e00", "carnator_size_discrepancy", "carnator_shape_discrepancy",
+    "carnator_compatibility_gate", "carnator_clopper_pearson_upper",
     "carnator_query_status", "carnator_status_string", "carnator_last_cuda_error",
     "carnator_kernel_launches", "carnator_version",
 ]
@@ -127,6 +129,17 @@ def lib() -> ctypes.CDLL:
     L.carnator_region_block_flags.argtypes = [vp, ps, ctypes.c_int32, ctypes.c_int32, vp, vp]
     L.carnator_sparse_attn_region.restype = ctypes.c_int
     L.carnator_sparse_attn_region.argtypes = [vp, vp, vp, vp, vp, vp, ps, vp, vp, vp, sz, vp]
+    dbl, pd = ctypes.c_double, ctypes.POINTER(ctypes.c_double)
+    L.carnator_delta_e00.restype = dbl
+    L.carnator_delta_e00.argtypes = [pd, pd]
+    L.carnator_size_discrepancy.restype = dbl
+    L.carnator_size_discrepancy.argtypes = [dbl, dbl]
+    L.carnator_shape_discrepancy.restype = dbl
+    L.carnator_shape_discrepancy.argtypes = [vp, ctypes.c_int32, ctypes.c_int32, vp, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+    L.carnator_compatibility_gate.restype = ctypes.c_int32
+    L.carnator_compatibility_gate.argtypes = [pd, pd, vp, ctypes.c_int32]
+    L.carnator_clopper_pearson_upper.restype = dbl
+    L.carnator_clopper_pearson_upper.argtypes = [ctypes.c_int32, ctypes.c_int32, dbl]
     L.carnator_query_status.restype = ctypes.c_int
     L.carnator_query_status.argtypes = [vp, vp]
     L.carnator_status_string.restype = ctypes.c_char_p
@@ -387,3 +400,37 @@ def sparse_attn_region(Q, K, V, mask, active_q, context_k, shape: Shape, O, LSE,
                                            ctypes.byref(shape), _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "carnator_sparse_attn_region")
     return ws
+
+
+# ---- host-side scalars (no GPU) ---------------------------------------------------------------------
+def delta_e00(lab_a, lab_b) -> float:
+    a = (ctypes.c_double * 3)(*[float(x) for x in lab_a])
+    b = (ctypes.c_double * 3)(*[float(x) for x in lab_b])
+    return float(lib().carnator_delta_e00(a, b))
+
+
+def size_discrepancy(area_q: float, area_j: float) -> float:
+    return float(lib().carnator_size_discrepancy(float(area_q), float(area_j)))
+
+
+def shape_discrepancy(m_q, m_j, resolution: int = 32) -> float:
+    """m_q, m_j: 2-D numpy uint8 indicators."""
+    import numpy as np
+    a = np.ascontiguousarray(m_q, dtype=np.uint8)
+    b = np.ascontiguousarray(m_j, dtype=np.uint8)
+    return float(lib().carnator_shape_discrepancy(a.ctypes.data, a.shape[0], a.shape[1], b.ctypes.data, b.shape[0], b.shape[1],
+                                                  int(resolution)))
+
+
+def compatibility_gate(d, tau, applicable=None) -> int:
+    n = len(d)
+    dd = (ctypes.c_double * n)(*[float(x) for x in d])
+    tt = (ctypes.c_double * n)(*[float(x) for x in tau])
+    ap = None
+    if applicable is not None:
+        ap = (ctypes.c_uint8 * n)(*[int(bool(x)) for x in applicable])
+    return int(lib().carnator_compatibility_gate(dd, tt, ap, n))
+
+
+def clopper_pearson_upper(unsafe: int, accepted: int, alpha: float) -> float:
+    return float(lib().carnator_clopper_pearson_upper(int(unsafe), int(accepted), float(alpha)))

@@ -13,6 +13,7 @@
 #include "attn_tcgen05.cuh"
 #include "block_mass_tcgen05.cuh"
 #include "regions.cuh"
+#include "compat_host.inl"
 
 using namespace carnator;
 
@@ -597,6 +598,41 @@ extern "C" carnator_status carnator_sparse_attn_region(const void* Q, const void
     st = compact_impl(mask, nullptr, active_q, context_k, s, ws, ws_bytes, stream);
     if (st != CARNATOR_OK) return st;
     return carnator_sparse_attn_compacted(Q, K, V, s, O, LSE, ws, ws_bytes, stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// host-side compatibility scalars and risk bound
+// ------------------------------------------------------------------------------------------------
+extern "C" double carnator_delta_e00(const double* lab_a, const double* lab_b) {
+    if (!lab_a || !lab_b) return NAN;
+    return carnator_host::delta_e00(lab_a, lab_b);
+}
+
+extern "C" double carnator_size_discrepancy(double area_q, double area_j) {
+    if (!(area_q > 0.0) || !(area_j > 0.0)) return NAN;
+    return std::fabs(std::log(area_q / area_j));
+}
+
+extern "C" double carnator_shape_discrepancy(const uint8_t* m_q, int32_t hq, int32_t wq, const uint8_t* m_j, int32_t hj,
+                                             int32_t wj, int32_t resolution) {
+    if (!m_q || !m_j || hq <= 0 || wq <= 0 || hj <= 0 || wj <= 0 || resolution <= 0) return NAN;
+    std::vector<uint8_t> a, b;
+    if (!carnator_host::bbox_normalize(m_q, hq, wq, resolution, a) || !carnator_host::bbox_normalize(m_j, hj, wj, resolution, b)) return NAN;
+    long inter = 0, na = 0, nb = 0;
+    for (size_t i = 0; i < a.size(); ++i) { inter += a[i] & b[i]; na += a[i]; nb += b[i]; }
+    return 1.0 - 2.0 * double(inter) / double(na + nb);
+}
+
+extern "C" int32_t carnator_compatibility_gate(const double* d, const double* tau, const uint8_t* applicable, int32_t n) {
+    if (!d || !tau || n < 0) return 0;
+    for (int k = 0; k < n; ++k)
+        if ((!applicable || applicable[k]) && !(d[k] <= tau[k])) return 0;
+    return 1;
+}
+
+extern "C" double carnator_clopper_pearson_upper(int32_t unsafe, int32_t accepted, double alpha) {
+    if (accepted <= 0 || unsafe < 0 || unsafe > accepted || !(alpha > 0.0 && alpha < 1.0)) return NAN;
+    return carnator_host::clopper_pearson_upper(unsafe, accepted, alpha);
 }
 
 // ------------------------------------------------------------------------------------------------
