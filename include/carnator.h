@@ -266,6 +266,30 @@ carnator_status carnator_sparse_attn_region(const void* Q, const void* K, const 
                                             void* ws, size_t ws_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
+ * Seeded self-attention expansion (Early-Signature localisation).
+ *
+ * Paper: Section 3.2 and Appendix "Evidence Region Construction" -- noun and background seed token sets
+ * I+ and I- are propagated through self-attention into the contrast score
+ *   S_i = Agg_h [ max_{u in I+} A_h[i,u] - max_{u in I-} A_h[i,u] ],   A_h[i,u] = exp(s_iu - LSE_i),
+ * A the dense self-attention weights.  Agg_h is taken as the mean over heads.  LSE is what a dense run of
+ * carnator_sparse_attn (all-ones mask) returns for the same Q and K.
+ *
+ *   Q, K      device, bf16, strides of `shape`;  LSE device, fp32 [B,H,N]
+ *   seeds     device, int32 [n_pos + n_neg] token indices in [0, N), positive set first, shared by all
+ *             heads and batch entries; an empty set contributes 0
+ *   per_head_opt  device, fp32 [B,H,N] or NULL: the per-head contrasts
+ *   contrast  device, fp32 [B,N], written
+ *   ws        device workspace, 256-byte aligned, >= carnator_seed_workspace_bytes
+ * ------------------------------------------------------------------------ */
+size_t carnator_seed_workspace_bytes(const carnator_shape* shape);
+
+carnator_status carnator_seed_expansion(const void* Q, const void* K, const float* LSE,
+                                        const int32_t* seeds, int32_t n_pos, int32_t n_neg,
+                                        const carnator_shape* shape,
+                                        float* per_head_opt, float* contrast,
+                                        void* ws, size_t ws_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
  * Host-side scalars of the reuse-validity gate and of its offline risk certificate.  No GPU work; all
  * pointers are HOST pointers; invalid arguments give NaN (0 for the gate).
  *

@@ -30,6 +30,7 @@ Pin status (tests/test_oracle_*.py):
   select_topk / select_cummass ...... pinned (stable sort, counts, order and minimality invariants)
   block_mass_exact / select_by_mass / build_connectivity_exact ... pinned (brute force, closed form, invariants)
   build_regions / fuse_latents / region_block_flags / attention_region_rows ... pinned (definitions by hand, closed forms)
+  seed_expansion ... pinned (dense softmax matrix by brute force, invariants)
   clopper_pearson_upper ... pinned (value printed in the paper, closed form for u = 0); delta_e00 / shape / size ... pinned (closed forms, invariants)
   fidelity of the pooled estimator to the true block attention mass: PARITY UNPINNED
   (the paper prints no mask, density or recall figure; it can only be reported, see tests).
@@ -464,6 +465,33 @@ def attention_region_rows(Qb, Kb, Vb, N, block_q, block_k, scale, mask, active_q
             O[r] = np.nan
             L[r] = np.nan
     return O, L
+
+
+# ==========================================================================
+# Seeded self-attention expansion (Section 3.2; Appendix "Evidence Region Construction")
+# ==========================================================================
+def seed_expansion(Qb, Kb, N, scale, seeds_pos, seeds_neg, lse: Optional[np.ndarray] = None):
+    """S_i = mean_h [ max_{u in I+} A_h[i,u] - max_{u in I-} A_h[i,u] ] with A the dense self-attention
+    weights (softmax over all N keys).  Returns (contrast [B, N], per_head [B, H, N]) in fp64.  ``lse``
+    [B, H, N] may be supplied; otherwise the softmax normaliser is computed here.  An empty seed set
+    contributes 0."""
+    B, H = Qb.shape[0], Qb.shape[1]
+    per_head = np.zeros((B, H, N))
+    sp = np.asarray(seeds_pos, dtype=np.int64)
+    sn = np.asarray(seeds_neg, dtype=np.int64)
+    for b in range(B):
+        for h in range(H):
+            q, k = _widen(Qb[b, h, :N]), _widen(Kb[b, h, :N])
+            if lse is None:
+                l = np.zeros(N)
+                for i0 in range(0, N, 1024):
+                    l[i0:i0 + 1024] = np.logaddexp.reduce(scale * (q[i0:i0 + 1024] @ k.T), axis=1)
+            else:
+                l = lse[b, h]
+            pos = np.exp(scale * (q @ k[sp].T) - l[:, None]).max(axis=1) if sp.size else 0.0
+            neg = np.exp(scale * (q @ k[sn].T) - l[:, None]).max(axis=1) if sn.size else 0.0
+            per_head[b, h] = pos - neg
+    return per_head.mean(axis=1), per_head
 
 
 # ==========================================================================

@@ -30,6 +30,7 @@ EXPORTS = [
     "carnator_sparse_attn_static",
     "carnator_regions_workspace_bytes", "carnator_build_regions", "carnator_fuse_latents",
     "carnator_region_block_flags", "carnator_sparse_attn_region",
+    "carnator_seed_workspace_bytes", "carnator_seed_expansion",
     "carnator_delta_e00", "carnator_size_discrepancy", "carnator_shape_discrepancy",
     "carnator_compatibility_gate", "carnator_clopper_pearson_upper",
     "carnator_query_status", "carnator_status_string", "carnator_last_cuda_error",
@@ -129,6 +130,10 @@ def lib() -> ctypes.CDLL:
     L.carnator_region_block_flags.argtypes = [vp, ps, ctypes.c_int32, ctypes.c_int32, vp, vp]
     L.carnator_sparse_attn_region.restype = ctypes.c_int
     L.carnator_sparse_attn_region.argtypes = [vp, vp, vp, vp, vp, vp, ps, vp, vp, vp, sz, vp]
+    L.carnator_seed_workspace_bytes.restype = sz
+    L.carnator_seed_workspace_bytes.argtypes = [ps]
+    L.carnator_seed_expansion.restype = ctypes.c_int
+    L.carnator_seed_expansion.argtypes = [vp, vp, vp, vp, ctypes.c_int32, ctypes.c_int32, ps, vp, vp, vp, sz, vp]
     dbl, pd = ctypes.c_double, ctypes.POINTER(ctypes.c_double)
     L.carnator_delta_e00.restype = dbl
     L.carnator_delta_e00.argtypes = [pd, pd]
@@ -400,6 +405,17 @@ def sparse_attn_region(Q, K, V, mask, active_q, context_k, shape: Shape, O, LSE,
                                            ctypes.byref(shape), _ptr(O), _ptr(LSE), _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "carnator_sparse_attn_region")
     return ws
+
+
+def seed_expansion(Q, K, LSE, seeds, n_pos: int, n_neg: int, shape: Shape, per_head=None, stream=None):
+    """carnator_seed_expansion.  seeds: int32 device tensor [n_pos + n_neg].  Returns contrast fp32 [B,N]."""
+    import torch
+    out = torch.empty((shape.B, shape.N), dtype=torch.float32, device=Q.device)
+    ws = _new_ws(int(lib().carnator_seed_workspace_bytes(ctypes.byref(shape))), Q.device)
+    st = lib().carnator_seed_expansion(_ptr(Q), _ptr(K), _ptr(LSE), _ptr(seeds), n_pos, n_neg, ctypes.byref(shape),
+                                       _ptr(per_head), _ptr(out), _ptr(ws), ws.numel(), _stream(stream))
+    _check(st, "carnator_seed_expansion")
+    return out
 
 
 # ---- host-side scalars (no GPU) ---------------------------------------------------------------------

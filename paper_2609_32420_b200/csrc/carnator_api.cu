@@ -13,6 +13,7 @@
 #include "attn_tcgen05.cuh"
 #include "block_mass_tcgen05.cuh"
 #include "regions.cuh"
+#include "seed_expand.cuh"
 #include "compat_host.inl"
 
 using namespace carnator;
@@ -598,6 +599,53 @@ extern "C" carnator_status carnator_sparse_attn_region(const void* Q, const void
     st = compact_impl(mask, nullptr, active_q, context_k, s, ws, ws_bytes, stream);
     if (st != CARNATOR_OK) return st;
     return carnator_sparse_attn_compacted(Q, K, V, s, O, LSE, ws, ws_bytes, stream);
+}
+
+// ------------------------------------------------------------------------------------------------
+// seeded self-attention expansion
+// ------------------------------------------------------------------------------------------------
+extern "C" size_t carnator_seed_workspace_bytes(const carnator_shape* s) {
+    if (check_shape(s, false) != CARNATOR_OK) return 0;
+    return align256(sizeof(WsHeader)) + align256(size_t(s->B) * s->H * s->N * 4);
+}
+
+extern "C" carnator_status carnator_seed_expansion(const void* Q, const void* K, const float* LSE, const int32_t* seeds,
+                                                   int32_t n_pos, int32_t n_neg, const carnator_shape* s,
+                                                   float* per_head_opt, float* contrast, void* ws, size_t ws_bytes,
+                                                   void* stream_) {
+    carnator_status st = check_shape(s, false);
+    if (st != CARNATOR_OK) return st;
+    if (!Q || !K || !LSE || !contrast || n_pos < 0 || n_neg < 0 || (n_pos + n_neg > 0 && !seeds)) return CARNATOR_ERR_INVALID_ARG;
+    if (!aligned(Q, 16) || !aligned(K, 16)) return CARNATOR_ERR_INVALID_ARG;
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    if (ws_bytes < carnator_seed_workspace_bytes(s)) return CARNATOR_ERR_WORKSPACE;
+    st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    SeedArgs a;
+    a.Q = static_cast<const __nv_bfloat16*>(Q); a.K = static_cast<const __nv_bfloat16*>(K);
+    for (int i = 0; i < 3; ++i) { a.qs[i] = s->q_stride[i]; a.ks[i] = s->k_stride[i]; }
+    a.LSE = LSE; a.seeds = seeds; a.n_pos = n_pos; a.n_neg = n_neg;
+    a.per_head = per_head_opt ? per_head_opt : reinterpret_cast<float*>(static_cast<char*>(ws) + align256(sizeof(WsHeader)));
+    a.B = s->B; a.H = s->H; a.N = s->N;
+    a.scale_log2 = effective_scale(s) * kLog2e;
+    dim3 grid(ceil_div(s->N, 128), s->H, s->B);
+    if (s->D == 128) {
+        const size_t smem = size_t(128 + 2 * 64) * (128 + 8) * 2;
+        st = allow_smem(seed_expand_kernel<128>, smem);
+        if (st != CARNATOR_OK) return st;
+        seed_expand_kernel<128><<<grid, 256, smem, stream>>>(a);
+    } else {
+        const size_t smem = size_t(128 + 2 * 64) * (64 + 8) * 2;
+        st = allow_smem(seed_expand_kernel<64>, smem);
+        if (st != CARNATOR_OK) return st;
+        seed_expand_kernel<64><<<grid, 256, smem, stream>>>(a);
+    }
+    LAUNCH_CHECK("seed_expand_kernel");
+    const int64_t n = int64_t(s->B) * s->N;
+    head_mean_kernel<<<unsigned((n + 255) / 256), 256, 0, stream>>>(a.per_head, s->B, s->H, s->N, contrast);
+    LAUNCH_CHECK("head_mean_kernel");
+    return CARNATOR_OK;
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -94,3 +94,31 @@ def test_region_attention_is_intersection_and_skips_inactive_rows():
         else:
             np.testing.assert_array_equal(O[r], O2[r])
             np.testing.assert_array_equal(L[r], L2[r])
+
+
+def test_seed_expansion_matches_dense_softmax_matrix_and_invariants():
+    """A taken from an explicitly materialised softmax matrix (every key), then the definition literally."""
+    import math
+    from tests.helpers import widen
+    rng = np.random.default_rng(30)
+    N, D, H = 40, 8, 3
+    Q, K = rand_bits(rng, (1, H, N, D)), rand_bits(rng, (1, H, N, D))
+    pos, neg = [3, 17, 22], [0, 5, 39, 11]
+    S, per_head = orc.seed_expansion(Q, K, N, 0.4, pos, neg)
+    q, k = widen(Q), widen(K)
+    exp_heads = np.zeros((H, N))
+    for h in range(H):
+        for i in range(N):
+            sc = [0.4 * float(q[0, h, i] @ k[0, h, j]) for j in range(N)]
+            den = sum(math.exp(v) for v in sc)
+            A = [math.exp(v) / den for v in sc]
+            exp_heads[h, i] = max(A[u] for u in pos) - max(A[u] for u in neg)
+    np.testing.assert_allclose(per_head[0], exp_heads, atol=1e-12)
+    np.testing.assert_allclose(S[0], exp_heads.mean(axis=0), atol=1e-12)
+    assert (np.abs(per_head) <= 1).all()
+    S_same, _ = orc.seed_expansion(Q, K, N, 0.4, pos, pos)
+    assert (S_same == 0).all()                                        # identical seed sets cancel
+    S_all, _ = orc.seed_expansion(Q, K, N, 0.4, list(range(N)), neg)
+    assert (S_all >= 0).all()                                         # max over every key dominates any subset
+    S_empty, ph = orc.seed_expansion(Q, K, N, 0.4, pos, [])
+    assert (ph > 0).all()
