@@ -1,0 +1,36 @@
+"""GPU parity of carnator_seed_expansion against the oracle, through the C ABI.  The LSE is the one a dense run
+of carnator_sparse_attn returns.  Values are attention probabilities in [0, 1]: pass if |d| <= 1e-3 * |ref| + 2e-6."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import carnator_oracle as orc
+from paper_2609_32420_b200 import carnator as cn
+from paper_2609_32420_b200 import workloads as wl
+from tests.gpu_util import to_dev
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,kw,n_pos,n_neg", [
+    ("wan1p3b_480p", dict(H=3, T=3), 150, 333),      # ragged seed counts (not multiples of 64), ragged N
+    ("cogvideox5b", dict(H=2, T=2), 64, 1),          # D = 64, text tokens present
+    ("wan1p3b_480p", dict(H=1, T=2), 5, 0),          # empty background set
+])
+def test_seed_expansion_matches_oracle(name, kw, n_pos, n_neg):
+    w = wl.shrunk(wl.get(name), **kw)
+    Qb, Kb = wl.gen_tensor(w, "Q"), wl.gen_tensor(w, "K")
+    Q, K = to_dev(Qb), to_dev(Kb)
+    V = torch.zeros_like(Q)
+    shape = cn.shape_of(w, Q, K, V)
+    ones = torch.ones((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device="cuda")
+    _, L, ws = cn.sparse_attn(Q, K, V, ones, None, shape)
+    assert cn.query_status(ws) == cn.OK
+    rng = np.random.default_rng(n_pos + n_neg)
+    tok = rng.choice(np.arange(w.n_text, w.N), size=n_pos + n_neg, replace=False).astype(np.int32)
+    seeds = torch.from_numpy(tok).cuda()
+    per_head = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device="cuda")
+    out = cn.seed_expansion(Q, K, L, seeds, n_pos, n_neg, cn.shape_of(w, Q, K), per_head=per_head)
+    S_ref, ph_ref = orc.seed_expansion(Qb, Kb, w.N, w.scale, tok[:n_pos], tok[n_pos:])
+    for got, ref in ((per_head.cpu().numpy(), ph_ref), (out.cpu().numpy(), S_ref)):
+        assert (np.abs(got - ref) <= 1e-3 * np.abs(ref) + 2e-6).all(), float(np.abs(got - ref).max())
