@@ -180,7 +180,7 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
 }
 
 // Shared-memory plan.  Q, and every K / V tile, is 128 rows x D held as D/64 boxes of 128 rows x 128 B
-// (128-byte swizzle).  K and V tiles travel through kStages-slot rings.
+// (128-byte swizzle).  K and V tiles travel through kStages-slot rings (separate rings, separate producers).
 template <int D>
 struct Cfg {
     static constexpr int kBoxes = D / 64;
@@ -212,6 +212,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     const int32_t* list = a.lists + (bh * a.nqb + I) * int64_t(a.nkb);
     const int q0 = I * kBlock;
 
+    if (T < 0) return;                      // skipped query block (region-restricted form): output untouched
     if (T == 0) {                           // nothing to attend to: O = 0, LSE = -inf
         if (tid < kBlock && q0 + tid < a.N) {
             __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(q0 + tid) * a.os[2];
@@ -282,8 +283,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 if (!mbar_wait(bar_kempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
                 }
+                const int J = list[i];
+                if (J < 0 || J >= a.nkb || (i > 0 && J <= list[i - 1])) {      // malformed list: stop before touching memory
+                    set_status(a.hdr, CARNATOR_ERR_DEVICE_CHECK, 21, i, blockIdx.x); *abortp = 1; break;
+                }
                 mbar_expect_tx(bar_kfull(s), C::kTileBytes);
-                const int key0 = list[i] * kBlock;
+                const int key0 = J * kBlock;
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
                     tma_load_4d(sK + s * C::kTileBytes + x * C::kBoxBytes, &mapK, bar_kfull(s), x * 64, key0, h, b);
@@ -304,8 +309,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 if (!mbar_wait(bar_vempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
                 }
+                const int J = list[i];
+                if (J < 0 || J >= a.nkb) { *abortp = 1; break; }                  // reported by the K producer
                 mbar_expect_tx(bar_vfull(s), C::kTileBytes);
-                const int key0 = list[i] * kBlock;
+                const int key0 = J * kBlock;
 #pragma unroll
                 for (int x = 0; x < C::kBoxes; ++x)
                     tma_load_4d(sV + s * C::kTileBytes + x * C::kBoxBytes, &mapV, bar_vfull(s), x * 64, key0, h, b);
