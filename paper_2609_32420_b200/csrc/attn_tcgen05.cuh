@@ -8,11 +8,14 @@
 //   warps 0-3  softmax group 0, warps 4-7 softmax group 1: the groups take the 128-key steps in turn; within
 //              a group warp w owns tensor-memory lanes 32w..32w+31 = query rows.  Both also run the epilogue.
 //   warp 8     TMA producer for Q and the K tiles (one lane)
-//   warp 9     tensor-memory allocation, issue of the Q K^T batches (one lane)
+//   warp 9     tensor-memory allocation, issue of every matrix product (one lane)
 //   warp 10    TMA producer for the V tiles (one lane)
-//   warp 11    issue of the P V batches (one lane)
+//   warp 11    idle
 // The third warpgroup gives most of its registers to the softmax groups (setmaxnreg), which hold a full
 // 128-column score row per thread.
+// One thread issues all the matrix products: two threads issuing at once each ran at half the rate, and the
+// pipe then executes in a known order.  Each batch ends in one tcgen05.commit (a commit costs the issuer about
+// as much as two MMAs): "S_g full" also releases the K slot, "P V done" also releases the V slot and P_g.
 // Tensor memory (512 columns): S0 | S1 (128 fp32 columns each, one per softmax group), P0 | P1 (64 columns
 // of packed bf16 each), O (D fp32 columns).  A group signals as soon as it has pulled its scores into
 // registers, so Q K^T of its next step runs underneath its own exponentials; P V is issued in step order.
@@ -33,7 +36,7 @@ constexpr int kRefSlots = 3;           // hand-over slots of the shared referenc
 constexpr int kStages = 2;             // ring slots for K tiles and for V tiles
 constexpr int kSoftmaxWarps = 8;       // two warpgroups taking the steps in turn
 constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // third warpgroup: two TMA producers, the MMA issuer, one idle warp
-constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10, kWarpMmaPV = 11;
+constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
 constexpr int kTmemCols = 512;         // S0 | S1 | P0 | P1 | O
 constexpr uint32_t kColP = 2 * kBlock; // packed bf16 probabilities: 64 columns per group
 constexpr uint32_t kColO = 2 * kBlock + 2 * 64;
@@ -54,6 +57,16 @@ __device__ __forceinline__ uint32_t mbar_try(uint32_t bar, uint32_t parity) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    return done;
+}
+// Non-blocking form for polling loops: try_wait may suspend the thread for a while when the phase is not complete.
+__device__ __forceinline__ uint32_t mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     return done;
@@ -79,12 +92,12 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
-// Warp-collective form: lane 0 waits (bounded), the outcome is broadcast; the shuffle orders the other
-// lanes' later reads after lane 0's acquire.
+// Warp-collective form.  Every lane tests the barrier (one broadcast read of shared memory, no divergence in the
+// common case that the phase is already complete); lanes that find it incomplete fall into the bounded wait.  The
+// vote makes the outcome uniform, reconverges the warp and orders the other lanes' later reads after the acquire.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0) {
-    int ok = 1;
-    if ((threadIdx.x & 31) == 0) ok = mbar_wait(bar, parity, abort_flag, sleep_ns) ? 1 : 0;
-    return __shfl_sync(0xffffffffu, ok, 0) != 0;
+    const bool ok = mbar_try(bar, parity) ? true : mbar_wait(bar, parity, abort_flag, sleep_ns);
+    return __all_sync(0xffffffffu, ok) != 0;
 }
 // One arrival per warp once every lane's earlier writes are ordered before it.
 __device__ __forceinline__ void mbar_arrive_warp(uint32_t bar) {
@@ -121,6 +134,22 @@ __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_
         "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
         ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
+// Same with the descriptors given as (low word, shared high word): the issuing thread keeps the low words in
+// registers and only adds a constant per instruction, which keeps its dependent instruction chain short.
+__device__ __forceinline__ void mma_ss_lo(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\tmov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_ts_lo(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\tsetp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     uint32_t r[32];
     asm volatile(
@@ -138,6 +167,11 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
 __device__ __forceinline__ float ex2_approx(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float y;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
     return y;
 }
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
@@ -228,11 +262,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     const uint32_t sK = smem_base + C::kOffK;
     const uint32_t sV = smem_base + C::kOffV;
     const uint32_t bars = smem_base + C::kOffBar;
-    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16, bar_drain2 = bars + 24;
+    const uint32_t bar_q = bars, bar_o = bars + 8, bar_drain = bars + 16;
     auto bar_kfull = [&](int s) { return bars + 32 + 8 * s; };       // up to 4 stages each
-    auto bar_kempty = [&](int s) { return bars + 64 + 8 * s; };
     auto bar_vfull = [&](int s) { return bars + 96 + 8 * s; };
-    auto bar_vempty = [&](int s) { return bars + 128 + 8 * s; };
     auto bar_sfull = [&](int s) { return bars + 160 + 8 * s; };      // S_g holds fresh scores
     auto bar_sfree = [&](int s) { return bars + 176 + 8 * s; };      // group g has read S_g into registers
     auto bar_pfull = [&](int s) { return bars + 192 + 8 * s; };      // P_g is complete
@@ -243,10 +275,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1); mbar_init(bar_drain2, 1);
+        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
         for (int s = 0; s < kStages; ++s) {
-            mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1);
-            mbar_init(bar_vfull(s), 1); mbar_init(bar_vempty(s), 1);
+            mbar_init(bar_kfull(s), 1); mbar_init(bar_vfull(s), 1);
         }
         for (int s = 0; s < kSBufs; ++s) {
             mbar_init(bar_sfull(s), 1); mbar_init(bar_pvdone(s), 1);
@@ -270,7 +301,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
     if (warp >= kSoftmaxWarps) {
     // Register budget: the producer / MMA warpgroup needs few registers and hands the rest to the softmax groups.
-    asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
+    // The CTA is launched with 384 x 168 registers; 256 x 216 + 128 x 72 uses exactly that.  A split that asks for
+    // more makes setmaxnreg.inc wait for registers that never come.
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 72;" ::: "memory");
     if (warp == kWarpTmaK) {
         // ================= TMA producer: Q once, then the K tiles =================
         if (lane == 0) {
@@ -279,8 +312,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
             int armed = -1;
             for (int i = 0; i < T; ++i) {
-                const int s = i % kStages;
-                if (!mbar_wait(bar_kempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
+                const int s = i % kStages, u = i - kStages;     // the slot is free once Q K^T of step u has completed
+                if (u >= 0 && !mbar_wait(bar_sfull(u & 1), uint32_t(u >> 1) & 1u, abortp, 100)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
                 }
                 const int J = list[i];
@@ -305,8 +338,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         if (lane == 0) {
             int armed = -1;
             for (int i = 0; i < T; ++i) {
-                const int s = i % kStages;
-                if (!mbar_wait(bar_vempty(s), (uint32_t(i / kStages) & 1u) ^ 1u, abortp, 200)) {
+                const int s = i % kStages, u = i - kStages;     // the slot is free once P V of step u has completed
+                if (u >= 0 && !mbar_wait(bar_pvdone(u & 1), uint32_t(u >> 1) & 1u, abortp, 100)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
                 }
                 const int J = list[i];
@@ -324,79 +357,77 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
         }
     } else if (warp == kWarpMma) {
-        // ================= MMA issuers =================
-        // Two issuing threads: warp 9 queues the Q K^T batches, warp 11 the P V batches.  The two chains touch
-        // disjoint tensor-memory columns (S_g vs P_g and O), so neither has to wait behind the other's queue.
+        // ================= MMA issuer =================
+        // One thread queues every matrix product and serves whichever is ready: Q K^T of the next step (its K tile
+        // has landed and the softmax group has taken the previous scores out of that S buffer) or P V of the oldest
+        // step whose probabilities are complete.  One commit per batch: the barrier that says "S_g is full" also
+        // frees the K slot, and the one that says "P V done" also frees the V slot and P_g.
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kBlock, kBlock, 0);
+            constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
+            // descriptor words that do not change: low word = (address >> 4) | leading offset; high word = stride
+            // offset | version | swizzle mode (see smem_desc)
+            const uint64_t dq = smem_desc(sQ, 16, 1024), dk = smem_desc(sK, 16, 1024), dv = smem_desc(sV, C::kBoxBytes, 1024);
+            const uint32_t q_lo = uint32_t(dq), k_lo0 = uint32_t(dk), hi_kmajor = uint32_t(dq >> 32);
+            const uint32_t v_lo0 = uint32_t(dv), hi_v = uint32_t(dv >> 32);
             bool ok = mbar_wait(bar_q, 0, abortp);
             if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
-            // S_g = Q K_i^T (g = i & 1): K-major operands, 16 elements of the head dimension per instruction
-            auto issue_qk = [&](int i) -> bool {
-                const int s = i % kStages, g = i & 1;
-                if (!mbar_wait(bar_kfull(s), uint32_t(i / kStages) & 1u, abortp, 20)) {
-                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, i, blockIdx.x); return false;
-                }
-                tc_fence_after();
+            int iq = 0, ip = 0;                          // next Q K^T step, next P V step
+            unsigned long long t_idle = 0;
+            uint32_t idle = 0;
+            while (ip < T && ok) {
+                bool progress = false;
+                if (iq < T) {
+                    const int s = iq % kStages, g = iq & 1;
+                    if (mbar_test(bar_kfull(s), uint32_t(iq / kStages) & 1u) &&
+                        (iq < 2 || mbar_test(bar_sfree(g), uint32_t((iq - 2) >> 1) & 1u))) {
+                        // S_g = Q K_i^T: K-major operands, 16 elements of the head dimension per instruction
+                        tc_fence_after();
+                        const uint32_t k_lo = k_lo0 + uint32_t(s) * (C::kTileBytes >> 4), d_s = tmem + g * kBlock;
 #pragma unroll
-                for (int kk = 0; kk < D / 16; ++kk) {
-                    const uint32_t off = (kk / 4) * C::kBoxBytes + (kk % 4) * 32;
-                    mma_ss(tmem + g * kBlock, smem_desc(sQ + off, 16, 1024),
-                           smem_desc(sK + s * C::kTileBytes + off, 16, 1024), idesc_qk, kk > 0);
+                        for (int kk = 0; kk < D / 16; ++kk) {
+                            const uint32_t off16 = ((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4;      // compile-time constant
+                            mma_ss_lo(d_s, q_lo + off16, k_lo + off16, hi_kmajor, idesc_qk, kk > 0 ? 1u : 0u);
+                        }
+                        tc_commit(bar_sfull(g));
+                        ++iq; progress = true;
+                    }
                 }
-                tc_commit(bar_sfull(g));
-                tc_commit(bar_kempty(s));
-                return true;
-            };
-            // Q K^T of step i may go as soon as group g has pulled S_g of step i-2 into registers
-            for (int i = 0; i < T && ok; ++i) {
-                if (i >= 2 && !mbar_wait(bar_sfree(i & 1), uint32_t((i - 2) >> 1) & 1u, abortp, 20)) {
-                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 14, i, blockIdx.x); ok = false; break;
+                if (ip < iq) {
+                    const int s = ip % kStages, g = ip & 1;
+                    if (mbar_test(bar_pfull(g), uint32_t(ip >> 1) & 1u) && mbar_test(bar_vfull(s), uint32_t(ip / kStages) & 1u)) {
+                        // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
+                        // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
+                        tc_fence_after();
+                        const uint32_t v_lo = v_lo0 + uint32_t(s) * (C::kTileBytes >> 4), p_t = tmem + kColP + g * 64, d_o = tmem + kColO;
+                        const uint32_t acc0 = ip > 0 ? 1u : 0u;
+#pragma unroll
+                        for (int kk = 0; kk < kBlock / 16; ++kk)
+                            mma_ts_lo(d_o, p_t + kk * 8, v_lo + kk * (2048 >> 4), hi_v, idesc_pv, kk > 0 ? 1u : acc0);
+                        tc_commit(bar_pvdone(g));
+                        ++ip; progress = true;
+                    }
                 }
-                ok = issue_qk(i);
+                if (progress) { idle = 0; continue; }
+                __nanosleep(20);                        // keep the polling from taking issue slots from the softmax warp on this scheduler
+                if ((++idle & 1023u) == 0) {             // nothing was ready: bounded, like every other wait
+                    if (*abortp) { ok = false; break; }
+                    const unsigned long long now = global_ns();
+                    if (idle == 1024u) t_idle = now;
+                    else if (now - t_idle > 2000000000ull) {
+                        set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 4, ip, blockIdx.x); *abortp = 1; ok = false; break;
+                    }
+                }
             }
+            if (ok) tc_commit(bar_o);
             if (*abortp) {      // make sure no MMA of this thread is still running before tensor memory is released
                 tc_commit(bar_drain);
                 mbar_wait(bar_drain, 0, abortp);
             }
         }
-    } else if (warp == kWarpMmaPV) {
-        if (lane == 0) {
-            constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
-            bool ok = true;
-            // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
-            // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
-            auto issue_pv = [&](int i) -> bool {
-                const int s = i % kStages, g = i & 1;
-                if (!mbar_wait(bar_vfull(s), uint32_t(i / kStages) & 1u, abortp, 20)) {
-                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 6, i, blockIdx.x); return false;
-                }
-                tc_fence_after();
-#pragma unroll
-                for (int kk = 0; kk < kBlock / 16; ++kk) {
-                    mma_ts(tmem + kColO, tmem + kColP + g * 64 + kk * 8,
-                           smem_desc(sV + s * C::kTileBytes + kk * 2048, C::kBoxBytes, 1024), idesc_pv, (i > 0) || (kk > 0));
-                }
-                tc_commit(bar_vempty(s));
-                tc_commit(bar_pvdone(g));
-                return true;
-            };
-            // P V in step order, each once P_g is complete
-            for (int i = 0; i < T && ok; ++i) {
-                if (!mbar_wait(bar_pfull(i & 1), uint32_t(i >> 1) & 1u, abortp, 20)) {
-                    set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 5, i, blockIdx.x); ok = false; break;
-                }
-                ok = issue_pv(i);
-            }
-            if (ok) tc_commit(bar_o);
-            if (*abortp) {
-                tc_commit(bar_drain2);
-                mbar_wait(bar_drain2, 0, abortp);
-            }
-        }
     }
     } else {
-        asm volatile("setmaxnreg.inc.sync.aligned.u32 232;" ::: "memory");
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 216;" ::: "memory");
         // ================= softmax + epilogue (warps 0-7) =================
         // Two warpgroups take the steps in turn (group g: steps g, g+2, ...), each with one warp per
         // tensor-memory lane quarter, so one group's exponentials run while the other group's scores are
@@ -410,13 +441,15 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         const int row = q0 + r_loc;
         float m_w = -INFINITY, l_w = 0.f;                           // this group's reference and partial row sum
         bool ok = true;
+        // lists ascend, so only the last listed block can be the ragged one: read it once, off the per-step path
+        const int nvalid_last = a.N - list[T - 1] * kBlock;
         for (int i = wg; i < T; i += 2) {
             const int rs = i % kRefSlots;
             const uint32_t sph = uint32_t(i >> 1) & 1u;
             ok = mbar_wait_warp(bar_sfull(wg), sph, abortp, 20);   // warp-uniform: the loads below are collective
             if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, i, blockIdx.x); break; }
             tc_fence_after();
-            const int nvalid = a.N - list[i] * kBlock;              // >= 1; < 128 only for a ragged last block
+            const int nvalid = (i == T - 1) ? nvalid_last : kBlock;      // >= 1; < 128 only for a ragged last block
             const uint32_t tS = tmem + lane_base + wg * kBlock;
             const uint32_t tP = tmem + lane_base + kColP + wg * 64;
             float s[4][32];
@@ -437,7 +470,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
             for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int e = 0; e < 32; ++e) mx4[e & 3] = fmaxf(mx4[e & 3], s[c][e]);
+                for (int e = 0; e < 32; e += 2) mx4[(e >> 1) & 3] = max3(mx4[(e >> 1) & 3], s[c][e], s[c][e + 1]);
             const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * a.scale_log2;
             // reference handed over from step i-1
             float r_prev = -INFINITY, r_now = mx;

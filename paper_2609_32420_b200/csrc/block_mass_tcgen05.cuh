@@ -14,6 +14,10 @@
 namespace carnator {
 namespace tc {
 
+constexpr int kMassSoftmaxWarps = 8;                        // two warpgroups taking the key blocks in turn
+constexpr int kMassThreads = (kMassSoftmaxWarps + 4) * 32;  // third warpgroup: TMA producer, MMA issuer, two idle warps
+constexpr int kMassWarpTma = 8, kMassWarpMma = 9;
+constexpr int kMassTmemCols = 512;
 constexpr int kMassSBufs = 4;      // score buffers (128 fp32 columns each)
 constexpr int kMassStages = 4;     // K tile ring
 
@@ -37,7 +41,7 @@ struct MassCfg {
 };
 
 template <int D>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kMassThreads, 1)
 block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK, const MassArgs a) {
     using C = MassCfg<D>;
     extern __shared__ unsigned char smem_dyn[];
@@ -73,9 +77,9 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             for (int s = 0; s < 4; ++s) mbar_init(bar_red(g, s), 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kWarpTmaK && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); }
-    if (warp == kWarpMma) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols) : "memory");
+    if (warp == kMassWarpTma && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); }
+    if (warp == kMassWarpMma) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kMassTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -83,9 +87,9 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
 
-    if (warp >= kSoftmaxWarps) {
+    if (warp >= kMassSoftmaxWarps) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
-    if (warp == kWarpTmaK) {
+    if (warp == kMassWarpTma) {
         // ================= TMA producer: Q once, then every K tile of the head =================
         if (lane == 0) {
             mbar_expect_tx(bar_q, C::kTileBytes);
@@ -109,7 +113,7 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                     mbar_wait(bar_kfull((armed - k) % kMassStages), uint32_t((armed - k) / kMassStages) & 1u, abortp);
             }
         }
-    } else if (warp == kWarpMma) {
+    } else if (warp == kMassWarpMma) {
         // ================= MMA issuer: S[i % 4] = Q K_i^T =================
         if (lane == 0) {
             constexpr uint32_t idesc_qk = instr_desc(kBlock, kBlock, 0);
@@ -191,9 +195,9 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
 
     tc_fence_before();
     __syncthreads();
-    if (warp == kWarpMma) {
+    if (warp == kMassWarpMma) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kMassTmemCols) : "memory");
     }
 }
 
@@ -210,10 +214,10 @@ inline carnator_status launch_block_mass(const void* Q, const void* K, const int
     cudaError_t e;
     if (D == 128) {
         e = cudaFuncSetAttribute(tc::block_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(tc::MassCfg<128>::kSmemBytes));
-        if (e == cudaSuccess) tc::block_mass_kernel<128><<<grid, tc::kThreads, tc::MassCfg<128>::kSmemBytes, stream>>>(mq, mk, a);
+        if (e == cudaSuccess) tc::block_mass_kernel<128><<<grid, tc::kMassThreads, tc::MassCfg<128>::kSmemBytes, stream>>>(mq, mk, a);
     } else {
         e = cudaFuncSetAttribute(tc::block_mass_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(tc::MassCfg<64>::kSmemBytes));
-        if (e == cudaSuccess) tc::block_mass_kernel<64><<<grid, tc::kThreads, tc::MassCfg<64>::kSmemBytes, stream>>>(mq, mk, a);
+        if (e == cudaSuccess) tc::block_mass_kernel<64><<<grid, tc::kMassThreads, tc::MassCfg<64>::kSmemBytes, stream>>>(mq, mk, a);
     }
     if (e == cudaSuccess) e = cudaGetLastError();
     if (e != cudaSuccess) { snprintf(err, errlen, "block_mass_kernel: %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
