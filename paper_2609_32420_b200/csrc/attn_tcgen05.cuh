@@ -40,6 +40,7 @@ constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
 constexpr int kTmemCols = 512;         // S0 | S1 | P0 | P1 | O
 constexpr uint32_t kColP = 2 * kBlock; // packed bf16 probabilities: 64 columns per group
 constexpr uint32_t kColO = 2 * kBlock + 2 * 64;
+constexpr int kRegsService = 72, kRegsSoftmax = 216;   // setmaxnreg targets (the literals in the kernel must match)
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8, well inside bf16/fp32 range
 
 // ---- small PTX wrappers -----------------------------------------------------------------------
@@ -635,6 +636,15 @@ inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const
     auto kern = tc::attn_tcgen05_kernel<D>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, int(C::kSmemBytes));
     if (e != cudaSuccess) { snprintf(err, errlen, "cudaFuncSetAttribute(tcgen05): %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
+    // The register hand-over inside the kernel only completes if the CTA owns enough registers: check what the
+    // compiler allocated instead of finding out on the device.
+    cudaFuncAttributes fa;
+    e = cudaFuncGetAttributes(&fa, kern);
+    if (e != cudaSuccess) { snprintf(err, errlen, "cudaFuncGetAttributes(tcgen05): %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
+    if (fa.numRegs * tc::kThreads < tc::kSoftmaxWarps * 32 * tc::kRegsSoftmax + 128 * tc::kRegsService) {
+        snprintf(err, errlen, "attn_tcgen05_kernel was built with %d registers per thread: too few for its setmaxnreg split", fa.numRegs);
+        return CARNATOR_ERR_UNSUPPORTED;
+    }
     dim3 grid(a.nqb, a.H, a.B);
     kern<<<grid, tc::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, a);
     e = cudaGetLastError();

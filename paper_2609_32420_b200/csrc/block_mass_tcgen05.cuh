@@ -212,6 +212,15 @@ inline carnator_status launch_block_mass(const void* Q, const void* K, const int
     }
     dim3 grid(a.nqb, a.H, a.B);
     cudaError_t e;
+    {   // the kernel's setmaxnreg split (40 / 232) needs 168 registers per thread at launch
+        cudaFuncAttributes fa;
+        e = (D == 128) ? cudaFuncGetAttributes(&fa, tc::block_mass_kernel<128>) : cudaFuncGetAttributes(&fa, tc::block_mass_kernel<64>);
+        if (e != cudaSuccess) { snprintf(err, errlen, "cudaFuncGetAttributes(block_mass): %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
+        if (fa.numRegs * tc::kMassThreads < tc::kMassSoftmaxWarps * 32 * 232 + 128 * 40) {
+            snprintf(err, errlen, "block_mass_kernel was built with %d registers per thread: too few for its setmaxnreg split", fa.numRegs);
+            return CARNATOR_ERR_UNSUPPORTED;
+        }
+    }
     if (D == 128) {
         e = cudaFuncSetAttribute(tc::block_mass_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(tc::MassCfg<128>::kSmemBytes));
         if (e == cudaSuccess) tc::block_mass_kernel<128><<<grid, tc::kMassThreads, tc::MassCfg<128>::kSmemBytes, stream>>>(mq, mk, a);
