@@ -200,6 +200,13 @@ carnator_status carnator_compacted_tiles(const carnator_shape* shape, const void
  * `arena` is a DEVICE buffer of at least carnator_*_host_arena_bytes that holds
  * the device copies and the workspace.  The calls copy in, run, copy out and
  * synchronise `stream` before returning.
+ * carnator_sparse_attn_host works through the heads in chunks of about 64 MB per
+ * tensor: the copy-in of one chunk, the kernels of the previous one and the
+ * copy-out of the one before run at the same time, on two copy streams that the
+ * library creates once per device (first call) and keeps; the kernels run on
+ * `stream`, after everything queued on it before the call.  One such call at a
+ * time per process (an internal lock serialises them).  Each chunk has its own
+ * workspace header inside the arena; the call returns the first failure.
  * ------------------------------------------------------------------------ */
 size_t carnator_attn_host_arena_bytes(const carnator_shape* shape);
 

@@ -1,4 +1,5 @@
 // C-ABI entry points of libcarnator: argument validation, workspace layout, kernel launches.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -401,12 +402,34 @@ extern "C" carnator_status carnator_compacted_tiles(const carnator_shape* s, con
 // host-buffer forms
 // ------------------------------------------------------------------------------------------------
 namespace {
+// The host-buffer attention call works through the heads in chunks, so that the copy-in of chunk k+1, the kernels of
+// chunk k and the copy-out of chunk k-1 overlap (PCIe is full duplex and the copy engines run beside the SMs).
+constexpr int kMaxHostChunks = 64;
+constexpr size_t kHostChunkBytes = size_t(64) << 20;     // target size of one tensor's share of a chunk
+
+struct HostChunks {
+    int heads;          // heads per chunk (the last chunk of a batch entry may be shorter)
+    int per_batch;      // chunks per batch entry
+    int count;          // per_batch * B
+};
+HostChunks host_chunks(const carnator_shape* s) {
+    const size_t per_head = size_t(s->N) * s->D * 2;
+    int hc = int(std::min<size_t>(size_t(s->H), std::max<size_t>(1, (kHostChunkBytes + per_head - 1) / per_head)));
+    while (int64_t(s->B) * ceil_div(s->H, hc) > kMaxHostChunks && hc < s->H) ++hc;
+    HostChunks c;
+    c.heads = hc;
+    c.per_batch = ceil_div(s->H, hc);
+    c.count = c.per_batch * s->B;
+    return c;
+}
+
 struct HostArena {
     char *Q, *K, *V, *O;
     float* LSE;
     uint8_t *mask, *rec;
-    void* ws;
-    size_t ws_bytes, bytes;
+    char* ws;                   // one workspace per chunk, ws_stride apart
+    size_t ws_stride, bytes;
+    HostChunks chunks;
 };
 HostArena attn_arena_layout(void* base, const carnator_shape* s) {
     HostArena a;
@@ -421,9 +444,10 @@ HostArena attn_arena_layout(void* base, const carnator_shape* s) {
     a.LSE = reinterpret_cast<float*>(p + off); off += align256(size_t(s->B) * s->H * s->N * 4);
     a.mask = reinterpret_cast<uint8_t*>(p + off); off += align256(size_t(s->B) * s->H * nqb * nkb);
     a.rec = reinterpret_cast<uint8_t*>(p + off); off += align256(size_t(s->B) * nqb);
+    a.chunks = host_chunks(s);
     a.ws = p + off;
-    a.ws_bytes = attn_ws_layout(nullptr, s->B, s->H, nqb, nkb).bytes;
-    off += a.ws_bytes;
+    a.ws_stride = align256(attn_ws_layout(nullptr, 1, a.chunks.heads, nqb, nkb).bytes);
+    off += a.ws_stride * a.chunks.count;
     a.bytes = off;
     return a;
 }
@@ -431,6 +455,80 @@ void contiguous_strides(carnator_shape* c) {
     const int64_t n = c->N, d = c->D, h = c->H;
     int64_t st[3] = {h * n * d, n * d, d};
     for (int i = 0; i < 3; ++i) c->q_stride[i] = c->k_stride[i] = c->v_stride[i] = c->o_stride[i] = st[i];
+}
+
+// Streams and events of the chunk pipeline: made once per device and kept.  One host-buffer attention call at a time
+// uses them (g_pipe_mu is held for the whole call).
+struct HostPipe {
+    bool ready = false;
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    cudaEvent_t ev_start = nullptr, ev_out = nullptr;
+    cudaEvent_t ev_in[kMaxHostChunks], ev_comp[kMaxHostChunks];
+};
+constexpr int kMaxPipeDevices = 32;
+std::mutex g_pipe_mu;
+HostPipe g_pipes[kMaxPipeDevices];
+
+carnator_status get_pipe(HostPipe** out) {
+    int dev = 0;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxPipeDevices) return CARNATOR_ERR_UNSUPPORTED;
+    HostPipe& p = g_pipes[dev];
+    if (!p.ready) {
+        CUDA_TRY(cudaStreamCreateWithFlags(&p.s_in, cudaStreamNonBlocking));
+        CUDA_TRY(cudaStreamCreateWithFlags(&p.s_out, cudaStreamNonBlocking));
+        CUDA_TRY(cudaEventCreateWithFlags(&p.ev_start, cudaEventDisableTiming));
+        CUDA_TRY(cudaEventCreateWithFlags(&p.ev_out, cudaEventDisableTiming));
+        for (int k = 0; k < kMaxHostChunks; ++k) {
+            CUDA_TRY(cudaEventCreateWithFlags(&p.ev_in[k], cudaEventDisableTiming));
+            CUDA_TRY(cudaEventCreateWithFlags(&p.ev_comp[k], cudaEventDisableTiming));
+        }
+        p.ready = true;
+    }
+    *out = &p;
+    return CARNATOR_OK;
+}
+
+// The body of the pipelined call; the caller drains all three streams whatever this returns.
+carnator_status attn_host_pipeline(const char* Q, const char* K, const char* V, const uint8_t* mask, const uint8_t* rec,
+                                   const carnator_shape& s, char* O, float* LSE, const HostArena& a, HostPipe& pipe,
+                                   cudaStream_t stream) {
+    const int nqb = ceil_div(s.N, s.block_q), nkb = ceil_div(s.N, s.block_k);
+    const size_t head_t = size_t(s.N) * s.D * 2, head_m = size_t(nqb) * nkb, head_l = size_t(s.N) * 4;
+    // everything queued on the caller's stream so far comes first
+    CUDA_TRY(cudaEventRecord(pipe.ev_start, stream));
+    CUDA_TRY(cudaStreamWaitEvent(pipe.s_in, pipe.ev_start, 0));
+    CUDA_TRY(cudaStreamWaitEvent(pipe.s_out, pipe.ev_start, 0));
+    if (rec) CUDA_TRY(cudaMemcpyAsync(a.rec, rec, size_t(s.B) * nqb, cudaMemcpyHostToDevice, pipe.s_in));
+    int k = 0;
+    for (int b = 0; b < s.B; ++b) {
+        for (int h0 = 0; h0 < s.H; h0 += a.chunks.heads, ++k) {
+            const int hc = std::min(a.chunks.heads, s.H - h0);
+            const size_t first = size_t(b) * s.H + h0;
+            const size_t ot = first * head_t, om = first * head_m, ol = first * head_l;
+            CUDA_TRY(cudaMemcpyAsync(a.Q + ot, Q + ot, hc * head_t, cudaMemcpyHostToDevice, pipe.s_in));
+            CUDA_TRY(cudaMemcpyAsync(a.K + ot, K + ot, hc * head_t, cudaMemcpyHostToDevice, pipe.s_in));
+            CUDA_TRY(cudaMemcpyAsync(a.V + ot, V + ot, hc * head_t, cudaMemcpyHostToDevice, pipe.s_in));
+            CUDA_TRY(cudaMemcpyAsync(a.mask + om, mask + om, hc * head_m, cudaMemcpyHostToDevice, pipe.s_in));
+            CUDA_TRY(cudaEventRecord(pipe.ev_in[k], pipe.s_in));
+            CUDA_TRY(cudaStreamWaitEvent(stream, pipe.ev_in[k], 0));
+            carnator_shape c = s;             // one batch entry, hc heads, strides of the whole tensor
+            c.B = 1;
+            c.H = hc;
+            carnator_status st = carnator_sparse_attn(a.Q + ot, a.K + ot, a.V + ot, a.mask + om, rec ? a.rec + size_t(b) * nqb : nullptr,
+                                                      &c, a.O + ot, reinterpret_cast<float*>(reinterpret_cast<char*>(a.LSE) + ol),
+                                                      a.ws + size_t(k) * a.ws_stride, a.ws_stride, stream);
+            if (st != CARNATOR_OK) return st;
+            CUDA_TRY(cudaEventRecord(pipe.ev_comp[k], stream));
+            CUDA_TRY(cudaStreamWaitEvent(pipe.s_out, pipe.ev_comp[k], 0));
+            CUDA_TRY(cudaMemcpyAsync(O + ot, a.O + ot, hc * head_t, cudaMemcpyDeviceToHost, pipe.s_out));
+            CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(LSE) + ol, reinterpret_cast<char*>(a.LSE) + ol, hc * head_l,
+                                     cudaMemcpyDeviceToHost, pipe.s_out));
+        }
+    }
+    CUDA_TRY(cudaEventRecord(pipe.ev_out, pipe.s_out));
+    CUDA_TRY(cudaStreamWaitEvent(stream, pipe.ev_out, 0));
+    return CARNATOR_OK;
 }
 }  // namespace
 
@@ -458,19 +556,23 @@ extern "C" carnator_status carnator_sparse_attn_host(const void* Q, const void* 
     st = check_device();
     if (st != CARNATOR_OK) return st;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const int nqb = ceil_div(s.N, s.block_q), nkb = ceil_div(s.N, s.block_k);
-    const size_t t = size_t(s.B) * s.H * s.N * s.D * 2;
-    CUDA_TRY(cudaMemcpyAsync(a.Q, Q, t, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(cudaMemcpyAsync(a.K, K, t, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(cudaMemcpyAsync(a.V, V, t, cudaMemcpyHostToDevice, stream));
-    CUDA_TRY(cudaMemcpyAsync(a.mask, mask, size_t(s.B) * s.H * nqb * nkb, cudaMemcpyHostToDevice, stream));
-    if (recompute_rows) CUDA_TRY(cudaMemcpyAsync(a.rec, recompute_rows, size_t(s.B) * nqb, cudaMemcpyHostToDevice, stream));
-    st = carnator_sparse_attn(a.Q, a.K, a.V, a.mask, recompute_rows ? a.rec : nullptr, &s, a.O, a.LSE, a.ws, a.ws_bytes, stream_);
+    std::lock_guard<std::mutex> lock(g_pipe_mu);
+    HostPipe* pipe = nullptr;
+    st = get_pipe(&pipe);
     if (st != CARNATOR_OK) return st;
-    CUDA_TRY(cudaMemcpyAsync(O, a.O, t, cudaMemcpyDeviceToHost, stream));
-    CUDA_TRY(cudaMemcpyAsync(LSE, a.LSE, size_t(s.B) * s.H * s.N * 4, cudaMemcpyDeviceToHost, stream));
-    CUDA_TRY(cudaStreamSynchronize(stream));
-    return carnator_query_status(a.ws, stream_);
+    st = attn_host_pipeline(static_cast<const char*>(Q), static_cast<const char*>(K), static_cast<const char*>(V), mask,
+                            recompute_rows, s, static_cast<char*>(O), LSE, a, *pipe, stream);
+    // nothing of this call may still be in flight when it returns, whatever happened above
+    const cudaError_t e1 = cudaStreamSynchronize(pipe->s_in), e2 = cudaStreamSynchronize(stream), e3 = cudaStreamSynchronize(pipe->s_out);
+    if (st != CARNATOR_OK) return st;
+    if (e1 != cudaSuccess) return cuda_fail(e1, "cudaStreamSynchronize(copy-in stream)");
+    if (e2 != cudaSuccess) return cuda_fail(e2, "cudaStreamSynchronize(stream)");
+    if (e3 != cudaSuccess) return cuda_fail(e3, "cudaStreamSynchronize(copy-out stream)");
+    for (int k = 0; k < a.chunks.count; ++k) {         // every chunk has its own status header; report the first failure
+        const carnator_status sk = carnator_query_status(a.ws + size_t(k) * a.ws_stride, stream_);
+        if (sk != CARNATOR_OK && st == CARNATOR_OK) st = sk;
+    }
+    return st;
 }
 
 extern "C" size_t carnator_build_host_arena_bytes(const carnator_shape* s_in, const carnator_build_params* p) {

@@ -198,3 +198,30 @@ def test_malformed_lists_are_reported_and_the_context_stays_usable():
     assert cn.query_status(ws) == cn.OK
     O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, N, 128, 128, 1.0 / np.sqrt(D), mask.cpu().numpy(), None)
     check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "after a reported list fault")
+
+
+@pytest.mark.parametrize("name,kw", [("wan1p3b_480p", {}), ("tiny", {"B": 2})], ids=["wan1p3b_two_head_chunks", "tiny_two_batch_entries"])
+def test_host_buffer_call_equals_device_call(name, kw):
+    """carnator_sparse_attn_host works through the heads in chunks on its own copy streams; the result must be
+    the device call's, bit for bit (same kernels, same inputs), with more than one chunk in flight."""
+    w = wl.get(name).replace(**kw) if kw else wl.get(name)
+    Qb, Kb, Vb = (wl.gen_tensor(w, t) for t in "QKV")
+    if w.Nbuf != w.N:
+        Qb, Kb, Vb = (np.ascontiguousarray(x[:, :, : w.N]) for x in (Qb, Kb, Vb))
+    mask = wl.gen_random_mask(w, density=0.3, seed=5)
+    rec = wl.gen_recompute_rows(w)
+    Q, K, V = to_dev(Qb), to_dev(Kb), to_dev(Vb)
+    shape = cn.shape_of(w, Q, K, V, None, attn_impl=cn.IMPL_AUTO)
+    O, L, ws = cn.sparse_attn(Q, K, V, torch.from_numpy(mask).cuda(), torch.from_numpy(rec).cuda(), shape)
+    assert cn.query_status(ws) == cn.OK, cn.last_cuda_error()
+    pin = [torch.from_numpy(x.view(np.int16)).pin_memory() for x in (Qb, Kb, Vb)]
+    hmask, hrec = torch.from_numpy(mask).pin_memory(), torch.from_numpy(rec).pin_memory()
+    hO = torch.full((w.B, w.H, w.N, w.D), 0x7FC0, dtype=torch.int16).pin_memory()
+    hL = torch.full((w.B, w.H, w.N), float("nan"), dtype=torch.float32).pin_memory()
+    hshape = cn.shape_of(w, attn_impl=cn.IMPL_AUTO)
+    arena = torch.empty(cn.attn_host_arena_bytes(hshape), dtype=torch.uint8, device="cuda")
+    for _ in range(2):                       # the second call reuses the cached streams and events
+        cn.sparse_attn_host(pin[0], pin[1], pin[2], hmask, hrec, hshape, hO, hL, arena)
+    O_dev = O[:, :, : w.N].contiguous().view(torch.int16).cpu()
+    assert torch.equal(hO, O_dev)
+    assert torch.equal(hL, L[:, :, : w.N].cpu())
