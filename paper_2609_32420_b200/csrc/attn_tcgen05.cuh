@@ -175,6 +175,26 @@ __device__ __forceinline__ float max3(float a, float b, float c) {
     asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
     return y;
 }
+// Two fp32 lanes per instruction (packed pair in a 64-bit register): halves the FMA-pipe instruction count of the
+// exponent arguments and of the row sums.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 __device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32]) {
@@ -378,6 +398,21 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             uint32_t idle = 0;
             while (ip < T && ok) {
                 bool progress = false;
+                if (ip < iq) {
+                    const int s = ip % kStages, g = ip & 1;
+                    if (mbar_test(bar_pfull(g), uint32_t(ip >> 1) & 1u) && mbar_test(bar_vfull(s), uint32_t(ip / kStages) & 1u)) {
+                        // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
+                        // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
+                        tc_fence_after();
+                        const uint32_t v_lo = v_lo0 + uint32_t(s) * (C::kTileBytes >> 4), p_t = tmem + kColP + g * 64, d_o = tmem + kColO;
+                        const uint32_t acc0 = ip > 0 ? 1u : 0u;
+#pragma unroll
+                        for (int kk = 0; kk < kBlock / 16; ++kk)
+                            mma_ts_lo(d_o, p_t + kk * 8, v_lo + kk * (2048 >> 4), hi_v, idesc_pv, kk > 0 ? 1u : acc0);
+                        tc_commit(bar_pvdone(g));
+                        ++ip; progress = true;
+                    }
+                }
                 if (iq < T) {
                     const int s = iq % kStages, g = iq & 1;
                     if (mbar_test(bar_kfull(s), uint32_t(iq / kStages) & 1u) &&
@@ -392,21 +427,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         }
                         tc_commit(bar_sfull(g));
                         ++iq; progress = true;
-                    }
-                }
-                if (ip < iq) {
-                    const int s = ip % kStages, g = ip & 1;
-                    if (mbar_test(bar_pfull(g), uint32_t(ip >> 1) & 1u) && mbar_test(bar_vfull(s), uint32_t(ip / kStages) & 1u)) {
-                        // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
-                        // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
-                        tc_fence_after();
-                        const uint32_t v_lo = v_lo0 + uint32_t(s) * (C::kTileBytes >> 4), p_t = tmem + kColP + g * 64, d_o = tmem + kColO;
-                        const uint32_t acc0 = ip > 0 ? 1u : 0u;
-#pragma unroll
-                        for (int kk = 0; kk < kBlock / 16; ++kk)
-                            mma_ts_lo(d_o, p_t + kk * 8, v_lo + kk * (2048 >> 4), hi_v, idesc_pv, kk > 0 ? 1u : acc0);
-                        tc_commit(bar_pvdone(g));
-                        ++ip; progress = true;
                     }
                 }
                 if (progress) { idle = 0; continue; }
@@ -512,22 +532,26 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             }
             if (m_w != r_now) { l_w *= ex2_approx(m_w - r_now); m_w = r_now; }   // first use: l_w = 0, exp2(-inf) = 0
             // P = exp2(s * scale - R_i): one FFMA + one MUFU per element, packed bf16 pairs over S's own columns
-            const float neg_m = -r_now;
-            float part[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint64_t neg_m2 = pack2(-r_now, -r_now), scale2 = pack2(a.scale_log2, a.scale_log2);
+            uint64_t part2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
-                    const float p0 = ex2_approx(fmaf(s[c][2 * e], a.scale_log2, neg_m));
-                    const float p1 = ex2_approx(fmaf(s[c][2 * e + 1], a.scale_log2, neg_m));
-                    part[e & 1] += p0;
-                    part[2 + (e & 1)] += p1;
+                    float x0, x1;
+                    unpack2(fma2(pack2(s[c][2 * e], s[c][2 * e + 1]), scale2, neg_m2), x0, x1);
+                    const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
+                    part2[e & 1] = add2(part2[e & 1], pack2(p0, p1));
                     pk[e] = pack_bf16(p0, p1);
                 }
                 tmem_st16(tP + c * 16, pk);
             }
-            l_w += (part[0] + part[1]) + (part[2] + part[3]);
+            {
+                float s0, s1, s2, s3;
+                unpack2(part2[0], s0, s1); unpack2(part2[1], s2, s3);
+                l_w += (s0 + s1) + (s2 + s3);
+            }
             tmem_wait_st();
             tc_fence_before();
             mbar_arrive_warp(bar_pfull(wg));
