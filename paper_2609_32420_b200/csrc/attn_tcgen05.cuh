@@ -7,7 +7,7 @@
 // Warp roles (384 threads = three warpgroups, one CTA per SM):
 //   warps 0-3  softmax group 0, warps 4-7 softmax group 1: the groups take the 128-key steps in turn; within
 //              a group warp w owns tensor-memory lanes 32w..32w+31 = query rows.  Both also run the epilogue.
-//   warp 8     TMA producer for Q and the K tiles (one lane)
+//   warp 8     TMA producer for the K tiles (one lane)
 //   warp 9     tensor-memory allocation, issue of every matrix product (one lane)
 //   warp 10    TMA producer for the V tiles (one lane)
 //   warp 11    idle
@@ -16,9 +16,13 @@
 // One thread issues all the matrix products: two threads issuing at once each ran at half the rate, and the
 // pipe then executes in a known order.  Each batch ends in one tcgen05.commit (a commit costs the issuer about
 // as much as two MMAs): "S_g full" also releases the K slot, "P V done" also releases the V slot and P_g.
-// Tensor memory (512 columns): S0 | S1 (128 fp32 columns each, one per softmax group), P0 | P1 (64 columns
-// of packed bf16 each), O (D fp32 columns).  A group signals as soon as it has pulled its scores into
-// registers, so Q K^T of its next step runs underneath its own exponentials; P V is issued in step order.
+// Tensor memory (512 columns): S0 | S1 (128 fp32 columns each, one per softmax group), P (64 columns of packed
+// bf16), Q (D / 2 columns of packed bf16), O (D fp32 columns).  The query tile is written there once by the
+// softmax groups (straight from global memory) and serves as the A operand of every Q K^T, so those products
+// read only the K tile from shared memory, whose bandwidth the TMA writes and the operand reads share.  A group
+// signals as soon as it has pulled its scores into registers, so Q K^T of its next step runs underneath its own
+// exponentials; it keeps its probabilities in registers until they are complete and stores them in one go, by
+// which time P V of the previous step has long read the one P buffer.  P V is issued in step order.
 // Every wait on an mbarrier is bounded; on expiry the role records CARNATOR_ERR_DEVICE_TIMEOUT in
 // the workspace header, raises a CTA-wide abort flag, and every role drains and returns.
 #pragma once
@@ -33,12 +37,13 @@ namespace tc {
 constexpr int kBlock = 128;            // query rows per CTA = keys per step
 constexpr int kSBufs = 2;              // score buffers in tensor memory, one per softmax group
 constexpr int kRefSlots = 3;           // hand-over slots of the shared reference maximum
-constexpr int kStages = 2;             // ring slots for K tiles and for V tiles
+constexpr int kStages = 3;             // ring slots for K tiles and for V tiles
 constexpr int kSoftmaxWarps = 8;       // two warpgroups taking the steps in turn
 constexpr int kThreads = (kSoftmaxWarps + 4) * 32;   // third warpgroup: two TMA producers, the MMA issuer, one idle warp
 constexpr int kWarpTmaK = 8, kWarpMma = 9, kWarpTmaV = 10;
 constexpr int kTmemCols = 512;         // S0 | S1 | P0 | P1 | O
-constexpr uint32_t kColP = 2 * kBlock; // packed bf16 probabilities: 64 columns per group
+constexpr uint32_t kColP = 2 * kBlock;        // packed bf16 probabilities: 64 columns, one buffer for both groups
+constexpr uint32_t kColQ = 2 * kBlock + 64;   // the query tile as packed bf16 pairs: D / 2 columns (A operand of Q K^T)
 constexpr uint32_t kColO = 2 * kBlock + 2 * 64;
 constexpr int kRegsService = 72, kRegsSoftmax = 216;   // setmaxnreg targets (the literals in the kernel must match)
 constexpr float kRescaleThreshold = 8.0f;   // log2 units: P stays below 2^8, well inside bf16/fp32 range
@@ -234,15 +239,14 @@ __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) 
     return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
 }
 
-// Shared-memory plan.  Q, and every K / V tile, is 128 rows x D held as D/64 boxes of 128 rows x 128 B
+// Shared-memory plan.  Every K / V tile is 128 rows x D held as D/64 boxes of 128 rows x 128 B
 // (128-byte swizzle).  K and V tiles travel through kStages-slot rings (separate rings, separate producers).
 template <int D>
 struct Cfg {
     static constexpr int kBoxes = D / 64;
     static constexpr uint32_t kBoxBytes = kBlock * 128;             // 128 rows x 128 B
     static constexpr uint32_t kTileBytes = kBoxes * kBoxBytes;      // one 128 x D bf16 tile
-    static constexpr uint32_t kOffQ = 0;
-    static constexpr uint32_t kOffK = kTileBytes;
+    static constexpr uint32_t kOffK = 0;
     static constexpr uint32_t kOffV = kOffK + kStages * kTileBytes;
     static constexpr uint32_t kOffBar = kOffV + kStages * kTileBytes;
     static constexpr uint32_t kSmemBytes = kOffBar + 512 + 1024;    // barriers + slack to align the base to 1 KiB
@@ -250,8 +254,7 @@ struct Cfg {
 
 template <int D>
 __global__ void __launch_bounds__(kThreads, 1)
-attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
-                    const __grid_constant__ CUtensorMap mapV, const AttnArgs a) {
+attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_constant__ CUtensorMap mapV, const AttnArgs a) {
     using C = Cfg<D>;
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_slot;
@@ -279,7 +282,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     }
 
     const uint32_t smem_base = (smem_u32(smem_dyn) + 1023u) & ~1023u;
-    const uint32_t sQ = smem_base + C::kOffQ;
     const uint32_t sK = smem_base + C::kOffK;
     const uint32_t sV = smem_base + C::kOffV;
     const uint32_t bars = smem_base + C::kOffBar;
@@ -296,7 +298,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 
     if (tid == 0) {
         abort_flag = 0;
-        mbar_init(bar_q, 1); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
+        mbar_init(bar_q, kSoftmaxWarps); mbar_init(bar_o, 1); mbar_init(bar_drain, 1);
         for (int s = 0; s < kStages; ++s) {
             mbar_init(bar_kfull(s), 1); mbar_init(bar_vfull(s), 1);
         }
@@ -309,7 +311,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         for (int q = 0; q < 4; ++q) mbar_init(bar_fin(q), 2);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == kWarpTmaK && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); }
+    if (warp == kWarpTmaK && lane == 0) prefetch_tmap(&mapK);
     if (warp == kWarpTmaV && lane == 0) prefetch_tmap(&mapV);
     if (warp == kWarpMma) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_slot)), "r"(kTmemCols) : "memory");
@@ -328,9 +330,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
     if (warp == kWarpTmaK) {
         // ================= TMA producer: Q once, then the K tiles =================
         if (lane == 0) {
-            mbar_expect_tx(bar_q, C::kTileBytes);
-#pragma unroll
-            for (int x = 0; x < C::kBoxes; ++x) tma_load_4d(sQ + x * C::kBoxBytes, &mapQ, bar_q, x * 64, q0, h, b);
             int armed = -1;
             for (int i = 0; i < T; ++i) {
                 const int s = i % kStages, u = i - kStages;     // the slot is free once Q K^T of step u has completed
@@ -349,7 +348,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                 armed = i;
             }
             if (*abortp) {      // copies in flight must land before the CTA gives its shared memory back
-                mbar_wait(bar_q, 0, abortp);
                 for (int k = 0; k < kStages && armed - k >= 0; ++k)
                     mbar_wait(bar_kfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, abortp);
             }
@@ -388,11 +386,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             constexpr uint32_t idesc_pv = instr_desc(kBlock, D, 1);
             // descriptor words that do not change: low word = (address >> 4) | leading offset; high word = stride
             // offset | version | swizzle mode (see smem_desc)
-            const uint64_t dq = smem_desc(sQ, 16, 1024), dk = smem_desc(sK, 16, 1024), dv = smem_desc(sV, C::kBoxBytes, 1024);
-            const uint32_t q_lo = uint32_t(dq), k_lo0 = uint32_t(dk), hi_kmajor = uint32_t(dq >> 32);
+            const uint64_t dk = smem_desc(sK, 16, 1024), dv = smem_desc(sV, C::kBoxBytes, 1024);
+            const uint32_t k_lo0 = uint32_t(dk), hi_kmajor = uint32_t(dk >> 32);
             const uint32_t v_lo0 = uint32_t(dv), hi_v = uint32_t(dv >> 32);
-            bool ok = mbar_wait(bar_q, 0, abortp);
+            bool ok = mbar_wait(bar_q, 0, abortp);        // the softmax groups have put the query tile into tensor memory
             if (!ok) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
+            tc_fence_after();
             int iq = 0, ip = 0;                          // next Q K^T step, next P V step
             unsigned long long t_idle = 0;
             uint32_t idle = 0;
@@ -404,7 +403,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
                         // O += P_i V_i : P_g from tensor memory (16 keys = 8 packed columns per instruction), V tile as the
                         // MN-major B operand (rows = keys, 64-element chunks of the head dimension one box apart)
                         tc_fence_after();
-                        const uint32_t v_lo = v_lo0 + uint32_t(s) * (C::kTileBytes >> 4), p_t = tmem + kColP + g * 64, d_o = tmem + kColO;
+                        const uint32_t v_lo = v_lo0 + uint32_t(s) * (C::kTileBytes >> 4), p_t = tmem + kColP, d_o = tmem + kColO;
                         const uint32_t acc0 = ip > 0 ? 1u : 0u;
 #pragma unroll
                         for (int kk = 0; kk < kBlock / 16; ++kk)
@@ -423,7 +422,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
 #pragma unroll
                         for (int kk = 0; kk < D / 16; ++kk) {
                             const uint32_t off16 = ((kk / 4) * C::kBoxBytes + (kk % 4) * 32) >> 4;      // compile-time constant
-                            mma_ss_lo(d_s, q_lo + off16, k_lo + off16, hi_kmajor, idesc_qk, kk > 0 ? 1u : 0u);
+                            mma_ts_lo(d_s, tmem + kColQ + kk * 8, k_lo + off16, hi_kmajor, idesc_qk, kk > 0 ? 1u : 0u);
                         }
                         tc_commit(bar_sfull(g));
                         ++iq; progress = true;
@@ -460,6 +459,33 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
         const int r_loc = quarter * 32 + lane;                      // query row within the tile
         const uint32_t lane_base = uint32_t(quarter * 32) << 16;
         const int row = q0 + r_loc;
+        {
+            // The query tile goes into tensor memory as the A operand of Q K^T (row = lane, two bf16 per column), so
+            // those products read only the K tile from shared memory.  Group g brings half of the head dimension.
+            const __nv_bfloat16* qp = a.Q + b * a.qs[0] + h * a.qs[1] + int64_t(row) * a.qs[2] + wg * (D / 2);
+#pragma unroll
+            for (int c = 0; c < D / 128; ++c) {
+                uint32_t r[32];
+#pragma unroll
+                for (int v = 0; v < 8; ++v) {
+                    const uint4 u = row < a.N ? *reinterpret_cast<const uint4*>(qp + c * 64 + v * 8) : make_uint4(0, 0, 0, 0);
+                    r[4 * v] = u.x; r[4 * v + 1] = u.y; r[4 * v + 2] = u.z; r[4 * v + 3] = u.w;
+                }
+                tmem_st32(tmem + lane_base + kColQ + wg * (D / 4) + c * 32, r);
+            }
+            if (D == 64) {
+                uint32_t r[16];
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    const uint4 u = row < a.N ? *reinterpret_cast<const uint4*>(qp + v * 8) : make_uint4(0, 0, 0, 0);
+                    r[4 * v] = u.x; r[4 * v + 1] = u.y; r[4 * v + 2] = u.z; r[4 * v + 3] = u.w;
+                }
+                tmem_st16(tmem + lane_base + kColQ + wg * 16, r);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            mbar_arrive_warp(bar_q);
+        }
         float m_w = -INFINITY, l_w = 0.f;                           // this group's reference and partial row sum
         bool ok = true;
         // lists ascend, so only the last listed block can be the ragged one: read it once, off the per-step path
@@ -472,7 +498,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             tc_fence_after();
             const int nvalid = (i == T - 1) ? nvalid_last : kBlock;      // >= 1; < 128 only for a ragged last block
             const uint32_t tS = tmem + lane_base + wg * kBlock;
-            const uint32_t tP = tmem + lane_base + kColP + wg * 64;
+            const uint32_t tP = tmem + lane_base + kColP;
             float s[4][32];
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, s[c]);
@@ -506,12 +532,12 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             r_pub[rs][r_loc] = r_now;
             mbar_arrive_warp(bar_ref(rs, quarter));
             // P_g is free again once P V of this group's previous step (i-2) has completed; in-order execution
-            // then also covers P V of step i-3
-            if (i >= 2) {
-                ok = mbar_wait_warp(bar_pvdone(wg), uint32_t((i - 2) >> 1) & 1u, abortp, 0);
-                if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 12, i, blockIdx.x); break; }
-            }
+            // then also covers P V of step i-3.  The probabilities are kept in registers until they are all there, so
+            // this wait comes after the exponentials, when that product has long finished; only the rescaling path,
+            // which needs the guarantee about step i-3 for the phase of the other group's barrier, takes it early.
+            bool p_free = i < 1;
             if (i > 0 && __any_sync(0xffffffffu, grow)) {
+                p_free = true;
                 // O must be quiescent: P V of step i-1 (the other group's) complete.  P V is issued in step order
                 // and that of step i cannot start before this group delivers P_i; the wait above has already
                 // established that P V of step i-3 is complete, so the phase of this barrier is unambiguous.
@@ -534,19 +560,24 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_const
             // P = exp2(s * scale - R_i): one FFMA + one MUFU per element, packed bf16 pairs over S's own columns
             const uint64_t neg_m2 = pack2(-r_now, -r_now), scale2 = pack2(a.scale_log2, a.scale_log2);
             uint64_t part2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
+            uint32_t pk[4][16];
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
 #pragma unroll
                 for (int e = 0; e < 16; ++e) {
                     float x0, x1;
                     unpack2(fma2(pack2(s[c][2 * e], s[c][2 * e + 1]), scale2, neg_m2), x0, x1);
                     const float p0 = ex2_approx(x0), p1 = ex2_approx(x1);
                     part2[e & 1] = add2(part2[e & 1], pack2(p0, p1));
-                    pk[e] = pack_bf16(p0, p1);
+                    pk[c][e] = pack_bf16(p0, p1);
                 }
-                tmem_st16(tP + c * 16, pk);
             }
+            if (!p_free) {      // the one P buffer is free once P V of step i-1 (the other group's) has read it
+                ok = mbar_wait_warp(bar_pvdone(wg ^ 1), uint32_t((i - 1) >> 1) & 1u, abortp, 0);
+                if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 12, i, blockIdx.x); break; }
+            }
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_st16(tP + c * 16, pk[c]);
             {
                 float s0, s1, s2, s3;
                 unpack2(part2[0], s0, s1); unpack2(part2[1], s2, s3);
@@ -654,7 +685,7 @@ inline bool tcgen05_supported(const carnator_shape* s) {
 }
 
 template <int D>
-inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv,
+inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mk, const CUtensorMap& mv,
                                  cudaStream_t stream, char* err, size_t errlen) {
     using C = tc::Cfg<D>;
     auto kern = tc::attn_tcgen05_kernel<D>;
@@ -670,7 +701,7 @@ inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const
         return CARNATOR_ERR_UNSUPPORTED;
     }
     dim3 grid(a.nqb, a.H, a.B);
-    kern<<<grid, tc::kThreads, C::kSmemBytes, stream>>>(mq, mk, mv, a);
+    kern<<<grid, tc::kThreads, C::kSmemBytes, stream>>>(mk, mv, a);
     e = cudaGetLastError();
     if (e != cudaSuccess) { snprintf(err, errlen, "attn_tcgen05_kernel: %s", cudaGetErrorString(e)); return CARNATOR_ERR_CUDA; }
     return CARNATOR_OK;
@@ -678,15 +709,14 @@ inline carnator_status launch_tc(const AttnArgs& a, const CUtensorMap& mq, const
 
 inline carnator_status launch_tcgen05(const AttnArgs& a, const carnator_shape* s, cudaStream_t stream,
                                       char* err, size_t errlen, long long* launches) {
-    CUtensorMap mq, mk, mv;
-    if (!tc::make_map(&mq, a.Q, a.B, a.H, a.N, s->D, a.qs, tc::kBlock) ||
-        !tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks, tc::kBlock) ||
+    CUtensorMap mk, mv;      // Q is read with plain loads (once per CTA, into tensor memory)
+    if (!tc::make_map(&mk, a.K, a.B, a.H, a.N, s->D, a.ks, tc::kBlock) ||
         !tc::make_map(&mv, a.V, a.B, a.H, a.N, s->D, a.vs, tc::kBlock)) {
         snprintf(err, errlen, "cuTensorMapEncodeTiled failed or is unavailable");
         return CARNATOR_ERR_CUDA;
     }
-    carnator_status st = (s->D == 128) ? launch_tc<128>(a, mq, mk, mv, stream, err, errlen)
-                                       : launch_tc<64>(a, mq, mk, mv, stream, err, errlen);
+    carnator_status st = (s->D == 128) ? launch_tc<128>(a, mk, mv, stream, err, errlen)
+                                       : launch_tc<64>(a, mk, mv, stream, err, errlen);
     if (st == CARNATOR_OK) *launches = 1;
     return st;
 }
