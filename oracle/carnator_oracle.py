@@ -533,6 +533,16 @@ def delta_e00(lab1, lab2) -> float:
     return float(np.sqrt((dLp / SL) ** 2 + (dCp / SC) ** 2 + (dHp / SH) ** 2 + RT * (dCp / SC) * (dHp / SH)))
 
 
+def context_discrepancy(labs_q, labs_j) -> float:
+    """d_context (Section 3.2, discrepancy vector): the largest CIEDE2000 difference between the target's and the
+    historical request's mean CIELAB colours over the shared nouns; 0 when no noun is shared.
+    labs_q[o], labs_j[o]: the (L*, a*, b*) of shared noun o in the two requests."""
+    d = 0.0
+    for cq, cj in zip(labs_q, labs_j):
+        d = max(d, delta_e00(cq, cj))
+    return d
+
+
 def bbox_normalized(m: np.ndarray, res: int) -> np.ndarray:
     """Crop a binary indicator to its tight support box and resample to res x res (nearest, cell centres)."""
     ys, xs = np.nonzero(m)
