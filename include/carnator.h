@@ -306,6 +306,8 @@ carnator_status carnator_seed_expansion(const void* Q, const void* K, const floa
  * Decision" -- one-sided Clopper-Pearson upper bound U_alpha(u, n) on the unsafe-reuse rate.
  *
  *   carnator_delta_e00            lab_a, lab_b: 3 doubles each (L*, a*, b*); k_L = k_C = k_H = 1
+ *   carnator_context_discrepancy  d_context = max over the n_shared shared nouns of the CIEDE2000 difference between
+ *                                 labs_q[3*o..3*o+2] and labs_j[3*o..3*o+2]; 0 when n_shared == 0
  *   carnator_size_discrepancy     positive tail-slice areas
  *   carnator_shape_discrepancy    binary indicators m_q [hq,wq], m_j [hj,wj]: each is cropped to its tight
  *                                 support box and resampled (cell centres, nearest) to resolution x resolution
@@ -314,6 +316,7 @@ carnator_status carnator_seed_expansion(const void* Q, const void* K, const floa
  *                                 P[Bin(n, p) <= u] = alpha (1 when u = n)
  * ------------------------------------------------------------------------ */
 double  carnator_delta_e00(const double* lab_a, const double* lab_b);
+double  carnator_context_discrepancy(const double* labs_q, const double* labs_j, int32_t n_shared);
 double  carnator_size_discrepancy(double area_q, double area_j);
 double  carnator_shape_discrepancy(const uint8_t* m_q, int32_t hq, int32_t wq,
                                    const uint8_t* m_j, int32_t hj, int32_t wj, int32_t resolution);

@@ -31,7 +31,7 @@ EXPORTS = [
     "carnator_regions_workspace_bytes", "carnator_build_regions", "carnator_fuse_latents",
     "carnator_region_block_flags", "carnator_sparse_attn_region",
     "carnator_seed_workspace_bytes", "carnator_seed_expansion",
-    "carnator_delta_e00", "carnator_size_discrepancy", "carnator_shape_discrepancy",
+    "carnator_delta_e00", "carnator_context_discrepancy", "carnator_size_discrepancy", "carnator_shape_discrepancy",
     "carnator_compatibility_gate", "carnator_clopper_pearson_upper",
     "carnator_query_status", "carnator_status_string", "carnator_last_cuda_error",
     "carnator_kernel_launches", "carnator_version",
@@ -137,6 +137,8 @@ def lib() -> ctypes.CDLL:
     dbl, pd = ctypes.c_double, ctypes.POINTER(ctypes.c_double)
     L.carnator_delta_e00.restype = dbl
     L.carnator_delta_e00.argtypes = [pd, pd]
+    L.carnator_context_discrepancy.restype = dbl
+    L.carnator_context_discrepancy.argtypes = [pd, pd, ctypes.c_int32]
     L.carnator_size_discrepancy.restype = dbl
     L.carnator_size_discrepancy.argtypes = [dbl, dbl]
     L.carnator_shape_discrepancy.restype = dbl
@@ -423,6 +425,16 @@ def delta_e00(lab_a, lab_b) -> float:
     a = (ctypes.c_double * 3)(*[float(x) for x in lab_a])
     b = (ctypes.c_double * 3)(*[float(x) for x in lab_b])
     return float(lib().carnator_delta_e00(a, b))
+
+
+def context_discrepancy(labs_q, labs_j) -> float:
+    """labs_q, labs_j: equally long sequences of (L*, a*, b*) triples, one per shared noun."""
+    n = len(labs_q)
+    if n != len(labs_j):
+        raise ValueError("one colour per shared noun on both sides")
+    a = (ctypes.c_double * (3 * n))(*[float(x) for c in labs_q for x in c])
+    b = (ctypes.c_double * (3 * n))(*[float(x) for c in labs_j for x in c])
+    return float(lib().carnator_context_discrepancy(a, b, n))
 
 
 def size_discrepancy(area_q: float, area_j: float) -> float:

@@ -758,6 +758,13 @@ extern "C" double carnator_delta_e00(const double* lab_a, const double* lab_b) {
     return carnator_host::delta_e00(lab_a, lab_b);
 }
 
+extern "C" double carnator_context_discrepancy(const double* labs_q, const double* labs_j, int32_t n_shared) {
+    if (n_shared < 0 || (n_shared > 0 && (!labs_q || !labs_j))) return NAN;
+    double d = 0.0;                                        // no shared noun: the dimension reads 0
+    for (int32_t o = 0; o < n_shared; ++o) d = std::max(d, carnator_host::delta_e00(labs_q + 3 * o, labs_j + 3 * o));
+    return d;
+}
+
 extern "C" double carnator_size_discrepancy(double area_q, double area_j) {
     if (!(area_q > 0.0) || !(area_j > 0.0)) return NAN;
     return std::fabs(std::log(area_q / area_j));

@@ -66,6 +66,35 @@ def test_delta_e00_closed_forms_and_invariants():
     assert abs(orc.delta_e00([50, e, 0], [50, -e, 0]) / (3 * e) - 1) < 1e-3
 
 
+PAIRS = os.path.join(os.path.dirname(os.path.abspath(__file__)), "golden", "ciede2000_published_pairs.txt")
+
+
+def _pairs():
+    rows = [[float(x) for x in ln.split()] for ln in open(PAIRS) if ln.strip() and not ln.startswith("#")]
+    assert len(rows) == 34
+    return rows
+
+
+def test_delta_e00_reproduces_the_published_check_pairs():
+    """Pins the hue half of the formula: T, the hue-difference and mean-hue wrap branches, and the rotation term
+    (sign and position), none of which the closed forms above reach."""
+    for i, r in enumerate(_pairs()):
+        assert abs(orc.delta_e00(r[0:3], r[3:6]) - r[6]) <= 1e-4, f"pair {i + 1}"
+        assert abs(orc.delta_e00(r[3:6], r[0:3]) - r[6]) <= 1e-4, f"pair {i + 1} swapped"
+        assert abs(cn.delta_e00(r[0:3], r[3:6]) - r[6]) <= 1e-4, f"pair {i + 1} (library)"
+
+
+def test_context_discrepancy_is_the_largest_difference_over_shared_nouns():
+    rows = _pairs()
+    assert orc.context_discrepancy([], []) == 0.0 == cn.context_discrepancy([], [])      # no shared noun
+    for sel in ([0], [3, 16, 24], [33, 18, 6, 20], list(range(34))):
+        q, j = [rows[i][0:3] for i in sel], [rows[i][3:6] for i in sel]
+        want = max(rows[i][6] for i in sel)                                              # published values
+        assert abs(orc.context_discrepancy(q, j) - want) <= 1e-4
+        assert abs(cn.context_discrepancy(q, j) - orc.context_discrepancy(q, j)) < 1e-9
+    assert math.isnan(cn.lib().carnator_context_discrepancy(None, None, 2))
+
+
 def test_shape_size_and_gate():
     yy, xx = np.mgrid[0:40, 0:60]
     disk = ((yy - 20) ** 2 + (xx - 30) ** 2 <= 15 ** 2).astype(np.uint8)
