@@ -75,16 +75,7 @@ def workload_from_args(args) -> wl.Workload:
 
 def gen_parallel(w, tensor, which):
     """All heads of one tensor, generated on a few host threads."""
-    from concurrent.futures import ThreadPoolExecutor
-    out = np.zeros((w.B, w.H, w.Nbuf, w.D), dtype=np.uint16)
-    jobs = [(b, h) for b in range(w.B) for h in range(w.H)]
-
-    def one(bh):
-        b, h = bh
-        out[b, h] = wl.gen_head(w, tensor, b, h, which)
-    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 1)) as ex:
-        list(ex.map(one, jobs))
-    return out
+    return wl.gen_tensor(w, tensor, which, threads=min(16, os.cpu_count() or 1))
 
 
 class ClockSampler:

@@ -22,6 +22,8 @@
  *   - Q, K, V, O are bf16 with the head dimension contiguous; the element
  *     strides of the (batch, head, token) axes are given in the shape record and
  *     must be multiples of 8 elements (16 bytes); base pointers 16-byte aligned.
+ *     A batch or head stride of 0 shares one tensor over that axis (e.g. K and V
+ *     common to all heads); such inputs run on the portable attention kernel.
  *   - Token order: text tokens first (n_text of them), then video tokens
  *     flattened frame-major (t, then grid row, then grid column).  Blocks are
  *     contiguous runs of block_q / block_k tokens of that order; the last block
@@ -58,7 +60,8 @@ typedef enum carnator_status {
 enum {
     CARNATOR_IMPL_AUTO = 0,      /* tcgen05 kernel where it supports the shape, else the portable kernel */
     CARNATOR_IMPL_PORTABLE = 1,  /* mma.sync kernel: any supported shape */
-    CARNATOR_IMPL_TCGEN05 = 2    /* TMA + tcgen05/TMEM kernel: block_q = block_k = 128; else CARNATOR_ERR_UNSUPPORTED */
+    CARNATOR_IMPL_TCGEN05 = 2    /* TMA + tcgen05/TMEM kernel: block_q = block_k = 128 and no zero K/V stride on a batch or head
+                                    axis longer than 1 (a tensor shared over heads); else CARNATOR_ERR_UNSUPPORTED */
 };
 
 /* Problem description shared by all calls. */
@@ -349,8 +352,11 @@ double  carnator_clopper_pearson_upper(int32_t unsafe, int32_t accepted, double 
  *     each call clears the header it relies on and rewrites every list entry it reads, so
  *     back-to-back calls on one stream are safe.  Two calls that overlap on the GPU (different
  *     streams, or different host threads without ordering) race on the array: order them.
- *   - The device status word of this form lives inside the array and is not exposed; use the
- *     workspace forms when bounded-wait diagnostics are needed.
+ *   - The device status word of this form lives at the start of the array.
+ *     carnator_static_status(stream) is carnator_query_status for it: it synchronises `stream`,
+ *     returns what kernels of earlier static-form calls on the current device reported
+ *     (CARNATOR_OK, CARNATOR_ERR_DEVICE_TIMEOUT or CARNATOR_ERR_DEVICE_CHECK) and clears the word.
+ *     It allocates nothing either.
  * ------------------------------------------------------------------------ */
 #define CARNATOR_STATIC_SCRATCH_BYTES (8u << 20)
 
@@ -358,6 +364,8 @@ carnator_status carnator_sparse_attn_static(const void* Q, const void* K, const 
                                             const uint8_t* mask, const uint8_t* recompute_rows,
                                             const carnator_shape* shape,
                                             void* O, float* LSE, void* stream);
+
+carnator_status carnator_static_status(void* stream);
 
 /* ------------------------------------------------------------------------
  * Status and diagnostics.

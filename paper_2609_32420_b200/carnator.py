@@ -27,7 +27,7 @@ EXPORTS = [
     "carnator_sparse_attn", "carnator_compacted_tiles",
     "carnator_attn_host_arena_bytes", "carnator_sparse_attn_host",
     "carnator_build_host_arena_bytes", "carnator_build_connectivity_host",
-    "carnator_sparse_attn_static",
+    "carnator_sparse_attn_static", "carnator_static_status",
     "carnator_regions_workspace_bytes", "carnator_build_regions", "carnator_fuse_latents",
     "carnator_region_block_flags", "carnator_sparse_attn_region",
     "carnator_seed_workspace_bytes", "carnator_seed_expansion",
@@ -120,6 +120,8 @@ def lib() -> ctypes.CDLL:
     L.carnator_build_connectivity_host.argtypes = [vp, vp, ps, pp, vp, vp, sz, vp]
     L.carnator_sparse_attn_static.restype = ctypes.c_int
     L.carnator_sparse_attn_static.argtypes = [vp, vp, vp, vp, vp, ps, vp, vp, vp]
+    L.carnator_static_status.restype = ctypes.c_int
+    L.carnator_static_status.argtypes = [vp]
     L.carnator_regions_workspace_bytes.restype = sz
     L.carnator_regions_workspace_bytes.argtypes = [ps]
     L.carnator_build_regions.restype = ctypes.c_int
@@ -359,6 +361,11 @@ def sparse_attn_static(Q, K, V, mask, recompute_rows, shape: Shape, O, LSE, stre
     st = lib().carnator_sparse_attn_static(_ptr(Q), _ptr(K), _ptr(V), _ptr(mask), _ptr(recompute_rows),
                                            ctypes.byref(shape), _ptr(O), _ptr(LSE), _stream(stream))
     _check(st, "carnator_sparse_attn_static")
+
+
+def static_status(stream=None) -> int:
+    """carnator_static_status: the device status word of the static-scratch form on the current device (read and cleared)."""
+    return int(lib().carnator_static_status(_stream(stream)))
 
 
 DTYPE_F32, DTYPE_BF16 = 0, 1

@@ -76,6 +76,19 @@ __global__ void __launch_bounds__(BQ * 2) attn_portable_kernel(AttnArgs a) {
     const int q0 = I * BQ;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, tig = lane & 3;
+    {
+        // The lists are only as good as the workspace they were read from: a count beyond nkb, an index outside
+        // [0, nkb) or a list that does not ascend stops this query block before anything is loaded.
+        int bad = count > a.nkb ? 1 : 0;
+        for (int i = tid; i < min(count, a.nkb); i += NT) {
+            const int J = list[i];
+            if (J < 0 || J >= a.nkb || (i > 0 && J <= list[i - 1])) bad = 1;
+        }
+        if (__syncthreads_or(bad)) {
+            if (tid == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_CHECK, 22, I, blockIdx.x);
+            return;
+        }
+    }
 
     const __nv_bfloat16* Qp = a.Q + b * a.qs[0] + h * a.qs[1];
     const __nv_bfloat16* Kp = a.K + b * a.ks[0] + h * a.ks[1];

@@ -101,6 +101,19 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return false;
 }
 
+// Wait used on the way out, after an abort: the copies or products this role still has in flight must land before
+// the CTA gives its shared and tensor memory back, so the abort flag does not end this wait; only time does.
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (uint32_t it = 0; it < (1u << 30); ++it) {
+        __nanosleep(100);
+        if (mbar_try(bar, parity)) return true;
+        if ((it & 255u) == 255u && global_ns() - t0 > 2000000000ull) break;
+    }
+    return false;
+}
+
 // Warp-collective form.  Every lane tests the barrier (one broadcast read of shared memory, no divergence in the
 // common case that the phase is already complete); lanes that find it incomplete fall into the bounded wait.  The
 // vote makes the outcome uniform, reconverges the warp and orders the other lanes' later reads after the acquire.
@@ -291,6 +304,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
     const int q0 = I * kBlock;
 
     if (T < 0) return;                      // skipped query block (region-restricted form): output untouched
+    if (T > a.nkb) {                        // a count that cannot come from compaction: stop before reading a list that long
+        if (tid == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_CHECK, 20, T, blockIdx.x);
+        return;
+    }
     if (T == 0) {                           // nothing to attend to: O = 0, LSE = -inf
         if (tid < kBlock && q0 + tid < a.N) {
             __nv_bfloat16* op = a.O + b * a.os[0] + h * a.os[1] + int64_t(q0 + tid) * a.os[2];
@@ -348,7 +365,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
     // more makes setmaxnreg.inc wait for registers that never come.
     asm volatile("setmaxnreg.dec.sync.aligned.u32 72;" ::: "memory");
     if (warp == kWarpTmaK) {
-        // ================= TMA producer: Q once, then the K tiles =================
+        // ================= TMA producer: the K tiles =================
         if (lane == 0) {
             int armed = -1;
             for (int i = 0; i < T; ++i) {
@@ -369,7 +386,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             }
             if (*abortp) {      // copies in flight must land before the CTA gives its shared memory back
                 for (int k = 0; k < kStages && armed - k >= 0; ++k)
-                    mbar_wait(bar_kfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, abortp);
+                    mbar_wait_drain(bar_kfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u);
             }
         }
     } else if (warp == kWarpTmaV) {
@@ -392,7 +409,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             }
             if (*abortp) {
                 for (int k = 0; k < kStages && armed - k >= 0; ++k)
-                    mbar_wait(bar_vfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, abortp);
+                    mbar_wait_drain(bar_vfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u);
             }
         }
     } else if (warp == kWarpMma) {
@@ -474,7 +491,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             if (ok) tc_commit_el(bar_o);
             if (__any_sync(0xffffffffu, *abortp != 0)) {      // make sure no MMA of this warp is still running before tensor memory is released
                 tc_commit_el(bar_drain);
-                mbar_wait_warp(bar_drain, 0, abortp);
+                mbar_wait_drain(bar_drain, 0);
+                __syncwarp();
             }
         }
     }
@@ -694,12 +712,12 @@ inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, in
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[4] = {cuuint64_t(D), cuuint64_t(N), cuuint64_t(H), cuuint64_t(B)};
-    // a stride of a size-1 axis is never used for addressing but must still be a valid value
+    // the stride of a size-1 axis is never used for addressing but must still be a valid value; a zero stride on a
+    // longer axis cannot be expressed (callers check tma_strides_ok before they get here)
     const cuuint64_t row = cuuint64_t(st[2]) * 2;
-    cuuint64_t s_h = (H > 1 || st[1] > 0) ? cuuint64_t(st[1]) * 2 : row * N;
-    cuuint64_t s_b = (B > 1 || st[0] > 0) ? cuuint64_t(st[0]) * 2 : s_h * H;
-    if (s_h == 0) s_h = row * N;
-    if (s_b == 0) s_b = s_h * H;
+    if ((H > 1 && st[1] <= 0) || (B > 1 && st[0] <= 0)) return false;
+    const cuuint64_t s_h = st[1] > 0 ? cuuint64_t(st[1]) * 2 : row * N;
+    const cuuint64_t s_b = st[0] > 0 ? cuuint64_t(st[0]) * 2 : s_h * H;
     cuuint64_t strides[3] = {row, s_h, s_b};
     cuuint32_t box[4] = {64, cuuint32_t(box_rows), 1, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -711,8 +729,15 @@ inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, in
 
 }  // namespace tc
 
+// A tensor map cannot express a zero stride, so a tensor that is shared over heads or batch entries (stride 0 on an
+// axis longer than 1) is not read through TMA: such shapes run on the portable kernel.
+inline bool tma_strides_ok(const carnator_shape* s, const int64_t st[3]) {
+    return (s->B == 1 || st[0] > 0) && (s->H == 1 || st[1] > 0);
+}
+
 inline bool tcgen05_supported(const carnator_shape* s) {
-    return s->block_q == tc::kBlock && s->block_k == tc::kBlock && (s->D == 64 || s->D == 128);
+    return s->block_q == tc::kBlock && s->block_k == tc::kBlock && (s->D == 64 || s->D == 128) &&
+           tma_strides_ok(s, s->k_stride) && tma_strides_ok(s, s->v_stride);
 }
 
 template <int D>

@@ -108,9 +108,9 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
                 armed = i;
             }
             if (*abortp) {      // copies in flight must land before the CTA gives its shared memory back
-                mbar_wait(bar_q, 0, abortp);
+                mbar_wait_drain(bar_q, 0);
                 for (int k = 0; k < kMassStages && armed - k >= 0; ++k)
-                    mbar_wait(bar_kfull((armed - k) % kMassStages), uint32_t((armed - k) / kMassStages) & 1u, abortp);
+                    mbar_wait_drain(bar_kfull((armed - k) % kMassStages), uint32_t((armed - k) / kMassStages) & 1u);
             }
         }
     } else if (warp == kMassWarpMma) {
@@ -139,7 +139,7 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             }
             // tensor memory may only be released once every MMA has retired
             tc_commit(bar_drain);
-            mbar_wait(bar_drain, 0, abortp);
+            mbar_wait_drain(bar_drain, 0);
         }
     }
     } else {

@@ -234,6 +234,7 @@ extern "C" carnator_status carnator_build_connectivity_exact(const void* Q, cons
     if (!aligned(Q, 16) || !aligned(K, 16) || !aligned(LSE, 4)) return CARNATOR_ERR_INVALID_ARG;
     if (block_mass_opt && !aligned(block_mass_opt, 4)) return CARNATOR_ERR_INVALID_ARG;
     if (s->block_q != tc::kBlock || s->block_k != tc::kBlock) return CARNATOR_ERR_UNSUPPORTED;
+    if (!tma_strides_ok(s, s->q_stride) || !tma_strides_ok(s, s->k_stride)) return CARNATOR_ERR_UNSUPPORTED;   // read through TMA
     const int nqb = ceil_div(s->N, s->block_q), nkb = ceil_div(s->N, s->block_k);
     if (nkb > kMaxKeyBlocksBuilder) return CARNATOR_ERR_UNSUPPORTED;
     if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
@@ -805,6 +806,23 @@ void* g_static_scratch_addr[kMaxDevices] = {nullptr};
 std::mutex g_static_mu;
 }  // namespace
 
+namespace {
+// Device address of the built-in array on the current device (looked up once per device, with that device current).
+carnator_status static_scratch_ptr(void** out) {
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return CARNATOR_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_scratch_addr[dev]) {
+        void* p = nullptr;
+        CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_addr[dev] = p;
+    }
+    *out = g_static_scratch_addr[dev];
+    return CARNATOR_OK;
+}
+}  // namespace
+
 extern "C" carnator_status carnator_sparse_attn_static(const void* Q, const void* K, const void* V,
                                                        const uint8_t* mask, const uint8_t* recompute_rows,
                                                        const carnator_shape* s, void* O, float* LSE, void* stream) {
@@ -819,21 +837,20 @@ extern "C" carnator_status carnator_sparse_attn_static(const void* Q, const void
     }
     st = check_device();
     if (st != CARNATOR_OK) return st;
-    int dev = -1;
-    CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= kMaxDevices) return CARNATOR_ERR_UNSUPPORTED;
     void* scratch = nullptr;
-    {
-        std::lock_guard<std::mutex> lock(g_static_mu);
-        if (!g_static_scratch_addr[dev]) {
-            void* p = nullptr;
-            CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));   // device address of the array on the current device
-            g_static_scratch_addr[dev] = p;
-        }
-        scratch = g_static_scratch_addr[dev];
-    }
+    st = static_scratch_ptr(&scratch);
+    if (st != CARNATOR_OK) return st;
     // carnator_sparse_attn clears the header and rewrites every list entry it later reads.
     return carnator_sparse_attn(Q, K, V, mask, recompute_rows, s, O, LSE, scratch, size_t(CARNATOR_STATIC_SCRATCH_BYTES), stream);
+}
+
+extern "C" carnator_status carnator_static_status(void* stream) {
+    carnator_status st = check_device();
+    if (st != CARNATOR_OK) return st;
+    void* scratch = nullptr;
+    st = static_scratch_ptr(&scratch);
+    if (st != CARNATOR_OK) return st;
+    return carnator_query_status(scratch, stream);       // the array starts with the same header as a workspace
 }
 
 // ------------------------------------------------------------------------------------------------

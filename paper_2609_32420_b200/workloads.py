@@ -198,12 +198,21 @@ def gen_head(w: Workload, tensor: str, b: int, h: int, which: str = "target") ->
 
 
 def gen_tensor(w: Workload, tensor: str, which: str = "target",
-               heads: Optional[Iterable[Tuple[int, int]]] = None) -> np.ndarray:
-    """bf16 bits [B, H, Nbuf, D].  With ``heads`` only those (b, h) are filled (others stay zero)."""
+               heads: Optional[Iterable[Tuple[int, int]]] = None, threads: int = 1) -> np.ndarray:
+    """bf16 bits [B, H, Nbuf, D].  With ``heads`` only those (b, h) are filled (others stay zero).
+    Every head has its own generator, so ``threads`` > 1 fills heads concurrently with identical bits."""
     out = np.zeros((w.B, w.H, w.Nbuf, w.D), dtype=np.uint16)
     todo = list(heads) if heads is not None else [(b, h) for b in range(w.B) for h in range(w.H)]
-    for (b, h) in todo:
-        out[b, h] = gen_head(w, tensor, b, h, which)
+
+    def one(bh):
+        out[bh[0], bh[1]] = gen_head(w, tensor, bh[0], bh[1], which)
+    if threads > 1 and len(todo) > 1:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(one, todo))
+    else:
+        for bh in todo:
+            one(bh)
     return out
 
 

@@ -84,6 +84,10 @@ def test_bad_pointers_strides_and_workspace():
     s4 = _shape()
     s4.attn_impl = 9
     assert call(s=s4) == cn.ERR_INVALID_ARG
+    s5 = _shape()                                              # K shared over the two heads: not expressible as a tensor map
+    s5.k_stride[1] = 0
+    s5.attn_impl = cn.IMPL_TCGEN05
+    assert call(s=s5) == cn.ERR_UNSUPPORTED
 
 
 def test_bad_build_params():

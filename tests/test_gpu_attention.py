@@ -5,6 +5,7 @@ configuration the benchmark times and compared on sampled (head, query block) ro
 which the oracle computes independently.
 """
 import dataclasses
+import os
 
 import numpy as np
 import pytest
@@ -141,54 +142,107 @@ def test_strided_inputs_and_rows_past_n_untouched(impl):
     check_attention(o_to_host(O[:, :, :N]), L.cpu().numpy(), O_ref, L_ref, "strided")
 
 
-FULL = [("wan1p3b_480p", None), ("cogvideox5b", None), ("wan14b_720p", None), ("hunyuan_720p", 0.10),
-        ("hunyuan_720p", 1.00)]      # keep ratio 1.0: all-ones mask, the dense check
+def test_keys_and_values_shared_over_heads():
+    """A head stride of 0 broadcasts one K / V over all heads (accepted input).  A tensor map cannot express it, so the
+    call must take the portable kernel and still match the oracle; asking for the tcgen05 kernel is refused."""
+    rng = np.random.default_rng(8)
+    B, H, N, D = 1, 3, 700, 128
+    Qb = rand_bits(rng, (B, H, N, D))
+    Kb1, Vb1 = rand_bits(rng, (B, 1, N, D)), rand_bits(rng, (B, 1, N, D))
+    Q, K, V = to_dev(Qb), to_dev(Kb1).expand(B, H, N, D), to_dev(Vb1).expand(B, H, N, D)
+    assert K.stride(1) == 0
+    nb = -(-N // 128)
+    mask = (rng.random((B, H, nb, nb)) < 0.5).astype(np.uint8)
+    shape = cn.make_shape(B, H, N, D, 0, 1, 1, N, 128, 128, Q, K, V, None, attn_impl=cn.IMPL_AUTO)
+    O, L, ws = cn.sparse_attn(Q, K, V, torch.from_numpy(mask).cuda(), None, shape)
+    assert cn.query_status(ws) == cn.OK
+    O_ref, L_ref = orc.attention_full(Qb, np.repeat(Kb1, H, axis=1), np.repeat(Vb1, H, axis=1), N, 128, 128, 1.0 / np.sqrt(D), mask, None)
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "K/V shared over heads")
+    shape.attn_impl = cn.IMPL_TCGEN05
+    with pytest.raises(cn.CarnatorError) as e:
+        cn.sparse_attn(Q, K, V, torch.from_numpy(mask).cuda(), None, shape)
+    assert e.value.status == cn.ERR_UNSUPPORTED
+
+
+# keep ratio 1.0: all-ones mask, the dense check; the HunyuanVideo-shaped layer is run at every density of its sweep
+FULL = [("wan1p3b_480p", None), ("cogvideox5b", None), ("wan14b_720p", None)] + \
+       [("hunyuan_720p", d) for d in wl.HUNYUAN_DENSITIES]
+
+_full_cache = {}
+
+
+def _full_inputs(name):
+    """Host bits and device tensors of one full-size workload, kept while consecutive cases use the same workload."""
+    if _full_cache.get("name") != name:
+        _full_cache.clear()
+        torch.cuda.empty_cache()
+        w = wl.get(name)
+        nthreads = min(16, os.cpu_count() or 1)
+        host = {t: wl.gen_tensor(w, t, threads=nthreads) for t in "QKV"}
+        dev = {t: to_dev(host[t]) for t in "QKV"}
+        dev["Qh"], dev["Kh"] = (to_dev(wl.gen_tensor(w, t, "history", threads=nthreads)) for t in "QK")
+        _full_cache.update(name=name, host=host, dev=dev)
+    return _full_cache["host"], _full_cache["dev"]
 
 
 @pytest.mark.parametrize("name,density", FULL, ids=[f[0] + ("" if f[1] is None else f"_{f[1]}") for f in FULL])
 def test_full_size_workload_sampled_rows(name, density):
-    """Whole layer at the benchmark's launch configuration (mask from the GPU builder on the
-    historical Q/K pair); sampled (head, query block) rows against the oracle."""
+    """Whole layer at the benchmark's launch configuration (mask from the GPU builder on the historical Q/K pair).
+    Every head is compared with the oracle on sampled query blocks: a recompute (forced-dense) block, the ragged
+    tail block, the shortest and the longest masked row, the text blocks where there are any, and a random one."""
     w = wl.get(name)
     if density is not None:
         w = w.replace(build=dataclasses.replace(w.build, keep_ratio=density))
-    heads = [(0, 0), (0, w.H - 1)]
-    Q, K, V = (to_dev(wl.gen_tensor(w, t)) for t in "QKV")
-    Qh, Kh = (to_dev(wl.gen_tensor(w, t, "history")) for t in "QK")
+    host, dev = _full_inputs(name)
+    Q, K, V = dev["Q"], dev["K"], dev["V"]
     shape = cn.shape_of(w, Q, K, V, None, attn_impl=cn.IMPL_AUTO)
-    mask_dev, _ = cn.build_connectivity(Qh, Kh, cn.shape_of(w, Qh, Kh), cn.params_of(w.build))
-    del Qh, Kh
+    mask_dev, _ = cn.build_connectivity(dev["Qh"], dev["Kh"], cn.shape_of(w, dev["Qh"], dev["Kh"]), cn.params_of(w.build))
     rec = wl.gen_recompute_rows(w)
     O, L, ws = cn.sparse_attn(Q, K, V, mask_dev, torch.from_numpy(rec).cuda(), shape)
     assert cn.query_status(ws) == cn.OK, cn.last_cuda_error()
     mask = mask_dev.cpu().numpy()
+    heads = [(b, h) for b in range(w.B) for h in range(w.H)]
     rows = pick_rows(mask, rec, w, heads, extra_per_head=1, seed=w.cfg)
-    # the oracle needs only the sampled heads on the host
-    Qb, Kb, Vb = wl.gen_qkv(w, heads=heads)
-    O_ref, L_ref = orc.attention_rows(Qb, Kb, Vb, w.N, w.block, w.block, w.scale, mask, rec, rows)
+    assert min(sum(1 for r in rows if r[:2] == bh) for bh in heads) >= 4
+    O_ref, L_ref = orc.attention_rows(host["Q"], host["K"], host["V"], w.N, w.block, w.block, w.scale, mask, rec, rows)
     O_g, L_g = gather_rows(O, L, rows, w)
     check_attention(O_g, L_g, O_ref, L_ref, f"{name} keep={w.build.keep_ratio}")
     if density == 1.0:
         assert bool((mask_dev == 1).all())
     # properties that hold at any size: every valid row finite, no row past N touched is checked above by shape
     assert torch.isfinite(O.float()).all() and torch.isfinite(L).all()
+    eff = (mask != 0) | (rec != 0)[:, None, :, None]
+    assert cn.compacted_tiles(shape, ws) == int(eff.sum())
 
 
-def test_malformed_lists_are_reported_and_the_context_stays_usable():
-    """Host-made fault: the compacted lists are overwritten between compaction and attention.  The tcgen05 kernel
-    must stop the affected query block, report CARNATOR_ERR_DEVICE_CHECK, and leave the device usable."""
+def test_full_size_inputs_are_released():
+    _full_cache.clear()
+    torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("impl", IMPLS, ids=IMPL_IDS)
+@pytest.mark.parametrize("fault", ["index", "count"])
+def test_malformed_lists_are_reported_and_the_context_stays_usable(impl, fault):
+    """Host-made fault: the compacted lists (or a count) are overwritten between compaction and attention.  Either
+    kernel must stop the affected query block before it loads anything, report CARNATOR_ERR_DEVICE_CHECK, and leave
+    the device usable."""
     rng = np.random.default_rng(21)
     B, H, N, D = 1, 1, 512, 128
     Qb, Kb, Vb = (rand_bits(rng, (B, H, N, D)) for _ in range(3))
     Q, K, V = to_dev(Qb), to_dev(Kb), to_dev(Vb)
-    shape = cn.make_shape(B, H, N, D, 0, 1, 1, N, 128, 128, Q, K, V, None, attn_impl=cn.IMPL_TCGEN05)
+    shape = cn.make_shape(B, H, N, D, 0, 1, 1, N, 128, 128, Q, K, V, None, attn_impl=impl)
     mask = torch.ones((B, H, 4, 4), dtype=torch.uint8, device="cuda")
     ws = cn.compact_mask(mask, None, shape)
     al = lambda x: (x + 255) // 256 * 256
     lists_off = 256 + 2 * al(4 * 4)                     # header | counts | order | lists
     lists = ws[lists_off: lists_off + 4 * 4 * 4].view(torch.int32)
     assert lists[:4].tolist() == [0, 1, 2, 3]
-    lists[1] = 1_000_000                                # row 0 now points far outside the key blocks
+    if fault == "index":
+        lists[1] = 1_000_000                            # row 0 now points far outside the key blocks
+    else:
+        counts = ws[256: 256 + 4 * 4].view(torch.int32)
+        assert counts.tolist() == [4, 4, 4, 4]
+        counts[2] = 9                                   # more listed blocks than there are key blocks
     O, L = cn.sparse_attn_compacted(Q, K, V, shape, ws)
     assert cn.query_status(ws) == cn.ERR_DEVICE_CHECK
     assert cn.query_status(ws) == cn.OK                 # reading the status clears it

@@ -5,6 +5,7 @@ within 1e-4 of the row's selection threshold; always-kept blocks must match; in 
 per-row count must match.  Pooled scores themselves are compared to 2e-5 absolute.
 """
 import dataclasses
+import os
 
 import numpy as np
 import pytest
@@ -98,15 +99,20 @@ def test_keep_ratio_one_is_all_ones():
     assert (mask_g == 1).all()
 
 
-FULL = ["wan1p3b_480p", "cogvideox5b", "wan14b_720p", "hunyuan_720p"]
+# the HunyuanVideo-shaped layer also at the ends of its density sweep
+FULL = [("wan1p3b_480p", None), ("cogvideox5b", None), ("wan14b_720p", None), ("hunyuan_720p", None),
+        ("hunyuan_720p", 0.05), ("hunyuan_720p", 0.50)]
 
 
-@pytest.mark.parametrize("name", FULL)
-def test_full_size_masks_on_sampled_heads(name):
+@pytest.mark.parametrize("name,keep", FULL, ids=[f[0] + ("" if f[1] is None else f"_{f[1]}") for f in FULL])
+def test_full_size_masks_on_sampled_heads(name, keep):
     """Full-size launch; the oracle checks two heads in full (every row, every block)."""
     w = wl.get(name)
+    if keep is not None:
+        w = w.replace(build=dataclasses.replace(w.build, keep_ratio=keep))
     heads = [(0, 1), (0, w.H - 2)]
-    Qb = wl.gen_tensor(w, "Q", "history")
-    Kb = wl.gen_tensor(w, "K", "history")
-    n_excused = _compare(w, Qb, Kb, heads=heads, what=name)
+    nthreads = min(16, os.cpu_count() or 1)
+    Qb = wl.gen_tensor(w, "Q", "history", threads=nthreads)
+    Kb = wl.gen_tensor(w, "K", "history", threads=nthreads)
+    n_excused = _compare(w, Qb, Kb, heads=heads, what=f"{name} keep={w.build.keep_ratio}")
     assert n_excused <= 8
