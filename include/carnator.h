@@ -107,6 +107,9 @@ typedef struct carnator_build_params {
  *   pooled_scores_opt  device, fp32 [B,H,nqb,nkb] contiguous or NULL; when given it
  *          receives S (and replaces the score area of the workspace)
  *   ws     device workspace, 256-byte aligned, >= carnator_build_workspace_bytes
+ * In top-k mode with nkb <= 1024, on layers large enough to fill the GPU, the three steps run as one persistent
+ * kernel (block sums on the tensor cores at HBM speed, fp32 scores and selection on chip beside them); otherwise,
+ * and in cumulative-mass mode, as three kernels with the scores held in the workspace.
  * Limits: nkb <= 4096.
  * ------------------------------------------------------------------------ */
 size_t carnator_build_workspace_bytes(const carnator_shape* shape, const carnator_build_params* params);
@@ -383,6 +386,10 @@ carnator_status carnator_static_status(void* stream);
  * the calling process so far (monotone counter).
  * ------------------------------------------------------------------------ */
 carnator_status carnator_query_status(void* ws, void* stream);
+/* Testing aid: which path carnator_build_connectivity takes in top-k mode.  0 = by size (the default), 1 = always
+ * the three separate kernels (pool, score, select), 2 = the persistent fused kernel wherever it supports the shape.
+ * Both compute the same pooled scores up to the order of the fp32 sums.  Process-wide. */
+void            carnator_debug_set_builder_path(int32_t path);
 const char*     carnator_status_string(carnator_status s);
 const char*     carnator_last_cuda_error(void);
 int64_t         carnator_kernel_launches(void);

@@ -33,7 +33,7 @@ EXPORTS = [
     "carnator_seed_workspace_bytes", "carnator_seed_expansion",
     "carnator_delta_e00", "carnator_context_discrepancy", "carnator_size_discrepancy", "carnator_shape_discrepancy",
     "carnator_compatibility_gate", "carnator_clopper_pearson_upper",
-    "carnator_query_status", "carnator_status_string", "carnator_last_cuda_error",
+    "carnator_query_status", "carnator_debug_set_builder_path", "carnator_status_string", "carnator_last_cuda_error",
     "carnator_kernel_launches", "carnator_version",
 ]
 
@@ -151,6 +151,8 @@ def lib() -> ctypes.CDLL:
     L.carnator_clopper_pearson_upper.argtypes = [ctypes.c_int32, ctypes.c_int32, dbl]
     L.carnator_query_status.restype = ctypes.c_int
     L.carnator_query_status.argtypes = [vp, vp]
+    L.carnator_debug_set_builder_path.restype = None
+    L.carnator_debug_set_builder_path.argtypes = [ctypes.c_int32]
     L.carnator_status_string.restype = ctypes.c_char_p
     L.carnator_status_string.argtypes = [ctypes.c_int]
     L.carnator_last_cuda_error.restype = ctypes.c_char_p
@@ -322,6 +324,14 @@ def compacted_tiles(shape: Shape, ws, stream=None) -> int:
 
 def query_status(ws, stream=None) -> int:
     return int(lib().carnator_query_status(_ptr(ws), _stream(stream)))
+
+
+BUILDER_AUTO, BUILDER_THREE_KERNELS, BUILDER_FUSED = 0, 1, 2
+
+
+def debug_set_builder_path(path: int) -> None:
+    """Testing aid: 0 = by size, 1 = three kernels, 2 = the fused persistent kernel where the shape allows it."""
+    lib().carnator_debug_set_builder_path(int(path))
 
 
 def attn_host_arena_bytes(shape: Shape) -> int:

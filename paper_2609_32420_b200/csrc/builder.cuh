@@ -394,4 +394,5 @@ __global__ void __launch_bounds__(256) select_topk_kernel(SelectArgs a, int rows
     }
 }
 
+
 }  // namespace carnator

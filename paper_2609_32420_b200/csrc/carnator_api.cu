@@ -12,6 +12,7 @@
 #include "compact.cuh"
 #include "attn_portable.cuh"
 #include "attn_tcgen05.cuh"
+#include "builder_fused.cuh"
 #include "block_mass_tcgen05.cuh"
 #include "regions.cuh"
 #include "seed_expand.cuh"
@@ -113,6 +114,58 @@ carnator_status allow_smem(K kernel, size_t bytes) {
 
 }  // namespace
 
+namespace {
+// Testing aid: 0 = choose by size, 1 = always the three kernels (pool, score, select), 2 = the persistent kernel
+// wherever it supports the shape; so that the two paths can be compared on any input.
+std::atomic<int> g_builder_path{0};
+
+carnator_status sm_count(int* out) {
+    static thread_local int cached_dev = -1, cached = 0;
+    int dev = -1;
+    CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != cached_dev) {
+        int n = 0;
+        CUDA_TRY(cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev));
+        cached_dev = dev; cached = n;
+    }
+    *out = cached;
+    return CARNATOR_OK;
+}
+
+constexpr size_t kMaxDynamicSmem = 227 * 1024;
+
+template <int D, int NPL, int R>
+carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap& mq, const CUtensorMap& mk, int nkb, int sms, cudaStream_t stream) {
+    const size_t smem = FusedSmem<D, R>::bytes(nkb);
+    carnator_status st = allow_smem(build_fused_kernel<D, NPL, R>, smem);
+    if (st != CARNATOR_OK) return st;
+    // the register hand-over inside the kernel (setmaxnreg) only completes if the CTA owns 256 x 32 + 512 x 104 registers
+    cudaFuncAttributes attr;
+    CUDA_TRY(cudaFuncGetAttributes(&attr, build_fused_kernel<D, NPL, R>));
+    if (attr.numRegs * kFusedThreads < 256 * 32 + 512 * 104) {
+        snprintf(g_cuda_error, sizeof(g_cuda_error), "build_fused_kernel was built with %d registers per thread: too few for its setmaxnreg split", attr.numRegs);
+        return CARNATOR_ERR_UNSUPPORTED;
+    }
+    build_fused_kernel<D, NPL, R><<<sms, kFusedThreads, smem, stream>>>(mq, mk, fa);
+    LAUNCH_CHECK("build_fused_kernel");
+    return CARNATOR_OK;
+}
+
+// a warp of the scoring group keeps NPL scores per row, two rows, in registers
+carnator_status launch_fused_builder(const FusedArgs& fa, const CUtensorMap& mq, const CUtensorMap& mk, int D, int nkb, int sms, cudaStream_t stream) {
+    if (D == 128) {
+        if (nkb <= 32 * 8) return launch_fused_r<128, 8, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+        if (nkb <= 32 * 24) return launch_fused_r<128, 24, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+        return launch_fused_r<128, 32, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+    }
+    if (nkb <= 32 * 8) return launch_fused_r<64, 8, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+    if (nkb <= 32 * 24) return launch_fused_r<64, 24, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+    return launch_fused_r<64, 32, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+}
+}  // namespace
+
+extern "C" void carnator_debug_set_builder_path(int32_t path) { g_builder_path.store(path == 1 || path == 2 ? path : 0); }
+
 // ------------------------------------------------------------------------------------------------
 // builder
 // ------------------------------------------------------------------------------------------------
@@ -143,9 +196,9 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     float* scores = pooled_scores_opt ? pooled_scores_opt : w.scores;
 
-    CUDA_TRY(cudaMemsetAsync(w.hdr, 0, sizeof(WsHeader), stream));
+    // header and the per-head pooled-block counters are contiguous: one clear
+    CUDA_TRY(cudaMemsetAsync(w.hdr, 0, align256(sizeof(WsHeader)) + align256(size_t(s->B) * s->H * 4), stream));
 
-    // M1
     PoolArgs pa;
     pa.X[0] = static_cast<const __nv_bfloat16*>(Q);
     pa.X[1] = static_cast<const __nv_bfloat16*>(K);
@@ -154,6 +207,39 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
     pa.nb[0] = nqb; pa.nb[1] = nkb;
     pa.out[0] = w.qbar; pa.out[1] = w.kbar;
     pa.N = s->N; pa.H = s->H;
+    SelectArgs sa;
+    sa.scores = scores; sa.mask = mask;
+    sa.nqb = nqb; sa.nkb = nkb; sa.npad = next_pow2(nkb); sa.H = s->H;
+    sa.mode = p->mode; sa.keep_ratio = p->keep_ratio; sa.mass = p->mass;
+    sa.count_includes_forced = p->count_includes_forced;
+    sa.k_all = topk_count_host(p->keep_ratio, nkb);
+    sa.values_are_mass = 0;
+    sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
+    sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
+
+    // The persistent kernel pays off once its scoring items fill the machine at least twice (its last items run after the
+    // pooling has ended); smaller layers take the three kernels.
+    int sms = 0;
+    st = sm_count(&sms);
+    if (st != CARNATOR_OK) return st;
+    const bool fused_able = p->mode == CARNATOR_MODE_TOPK && nkb <= 32 * 32 && tma_strides_ok(s, s->q_stride) && tma_strides_ok(s, s->k_stride);
+    const bool fused_pays = int64_t(s->B) * s->H * ceil_div(nqb, kFusedRows) >= 2 * int64_t(sms);
+    const int choice = g_builder_path.load();
+    if (fused_able && (choice == 2 || (choice == 0 && fused_pays))) {
+        // one persistent kernel: pooling, pooled scores and selection; the scores stay on chip
+        FusedArgs fa;
+        fa.pool = pa; fa.sel = sa;
+        fa.scores_out = pooled_scores_opt; fa.done = w.done; fa.hdr = w.hdr;
+        fa.B = s->B; fa.scale = effective_scale(s);
+        CUtensorMap mq, mk;      // one box = 64 elements x one block of tokens; rows >= N read as zero
+        if (!tc::make_map(&mq, Q, s->B, s->H, s->N, s->D, s->q_stride, s->block_q) ||
+            !tc::make_map(&mk, K, s->B, s->H, s->N, s->D, s->k_stride, s->block_k)) {
+            snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed or is unavailable");
+            return CARNATOR_ERR_CUDA;
+        }
+        return launch_fused_builder(fa, mq, mk, s->D, nkb, sms, stream);
+    }
+    // M1
     {
         dim3 grid(nqb > nkb ? nqb : nkb, s->H, 2 * s->B);
         if (s->D == 128) pool_kernel<128><<<grid, 256, 0, stream>>>(pa);
@@ -170,15 +256,6 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
     }
     // M3
     {
-        SelectArgs sa;
-        sa.scores = scores; sa.mask = mask;
-        sa.nqb = nqb; sa.nkb = nkb; sa.npad = next_pow2(nkb); sa.H = s->H;
-        sa.mode = p->mode; sa.keep_ratio = p->keep_ratio; sa.mass = p->mass;
-        sa.count_includes_forced = p->count_includes_forced;
-        sa.k_all = topk_count_host(p->keep_ratio, nkb);
-        sa.values_are_mass = 0;
-        sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
-        sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
         if (p->mode == CARNATOR_MODE_TOPK) {
             // register-resident selection, one warp per row
             const int rows = s->B * s->H * nqb;

@@ -17,7 +17,8 @@ struct WsHeader {
     int32_t status;              // carnator_status set by kernels (0 = ok); first error wins
     int32_t info[3];             // where a bounded wait gave up / which check failed
     unsigned long long tiles;    // evaluated (query block, key block) pairs after compaction
-    int32_t pad[58];
+    int32_t work[4];             // work-item counters of persistent kernels (zeroed with the header)
+    int32_t pad[54];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 
@@ -46,9 +47,10 @@ inline AttnWs attn_ws_layout(void* base, int B, int H, int nqb, int nkb) {
     return w;
 }
 
-// Layout of the builder workspace: header | qbar | kbar | scores.
+// Layout of the builder workspace: header | pooled-blocks counters | qbar | kbar | scores.
 struct BuildWs {
     WsHeader* hdr;
+    int32_t* done;   // [B,H]  pooled blocks of each head written so far (fused builder; zeroed together with the header)
     float* qbar;     // [B,H,nqb,D]
     float* kbar;     // [B,H,nkb,D]
     float* scores;   // [B,H,nqb,nkb]
@@ -60,6 +62,7 @@ inline BuildWs build_ws_layout(void* base, int B, int H, int nqb, int nkb, int D
     char* p = static_cast<char*>(base);
     size_t off = 0;
     w.hdr = reinterpret_cast<WsHeader*>(p + off);           off += align256(sizeof(WsHeader));
+    w.done = reinterpret_cast<int32_t*>(p + off);           off += align256(size_t(B) * H * 4);
     w.qbar = reinterpret_cast<float*>(p + off);             off += align256(size_t(B) * H * nqb * D * 4);
     w.kbar = reinterpret_cast<float*>(p + off);             off += align256(size_t(B) * H * nkb * D * 4);
     w.scores = reinterpret_cast<float*>(p + off);           off += align256(size_t(B) * H * nqb * size_t(nkb) * 4);
@@ -71,6 +74,12 @@ __device__ inline void set_status(WsHeader* hdr, int32_t code, int32_t i0, int32
     if (atomicCAS(&hdr->status, 0, code) == 0) {
         hdr->info[0] = i0; hdr->info[1] = i1; hdr->info[2] = i2;
     }
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
 }
 
 // Token geometry used by the always-kept rule of the builder.

@@ -49,18 +49,33 @@ def _compare(w, Qb, Kb, heads=None, what=""):
     return check_mask(mask_g, mask_r, scores_r, theta, F, topk_mode=(w.build.mode == wl.MODE_TOPK), what=what)
 
 
-def test_tiny_topk():
+PATHS = [cn.BUILDER_THREE_KERNELS, cn.BUILDER_FUSED]
+PATH_IDS = ["three_kernels", "fused"]
+
+
+@pytest.fixture
+def builder_path(request):
+    """Small layers would take the three kernels by size; the parity cases below run on both paths."""
+    cn.debug_set_builder_path(request.param)
+    yield request.param
+    cn.debug_set_builder_path(cn.BUILDER_AUTO)
+
+
+@pytest.mark.parametrize("builder_path", PATHS, ids=PATH_IDS, indirect=True)
+def test_tiny_topk(builder_path):
     w = wl.get("tiny")
     Qb, Kb, _ = wl.gen_qkv(w)
     _compare(w, Qb, Kb, what="tiny")
 
 
+@pytest.mark.parametrize("builder_path", PATHS, ids=PATH_IDS, indirect=True)
 @pytest.mark.parametrize("name,kw", [
     ("wan1p3b_480p", dict(H=2, T=3)),
     ("cogvideox5b", dict(H=3, T=2)),
     ("hunyuan_720p", dict(H=2, T=1)),
+    ("hunyuan_720p", dict(H=2, T=28)),         # nkb = 790: four score tiles per row, 32 keys per lane
 ])
-def test_midsize_window_text_rules(name, kw):
+def test_midsize_window_text_rules(name, kw, builder_path):
     w = wl.shrunk(wl.get(name), **kw)
     Qb, Kb, _ = wl.gen_qkv(w, "history")
     _compare(w, Qb, Kb, what=name)
@@ -77,7 +92,8 @@ def test_cumulative_mass_mode(name, kw, mass):
     _compare(w, Qb, Kb, what=f"{name} cummass {mass}")
 
 
-def test_ties_are_broken_by_lower_block_index():
+@pytest.mark.parametrize("builder_path", PATHS, ids=PATH_IDS, indirect=True)
+def test_ties_are_broken_by_lower_block_index(builder_path):
     """Identical key blocks give identical pooled scores: the lower index must win, exactly as the oracle does."""
     w = wl.shrunk(wl.get("wan1p3b_480p"), H=1, T=2).replace(
         build=wl.BuildParams(keep_ratio=0.3, window_frames=-1))
@@ -91,12 +107,43 @@ def test_ties_are_broken_by_lower_block_index():
     np.testing.assert_array_equal(mask_g[..., :full], mask_r[..., :full])
 
 
-def test_keep_ratio_one_is_all_ones():
+@pytest.mark.parametrize("builder_path", PATHS, ids=PATH_IDS, indirect=True)
+def test_keep_ratio_one_is_all_ones(builder_path):
     w = wl.shrunk(wl.get("hunyuan_720p"), H=1, T=1).replace()
     w = w.replace(build=dataclasses.replace(w.build, keep_ratio=1.0))
     Qb, Kb, _ = wl.gen_qkv(w, "history")
     mask_g, _ = _gpu(w, Qb, Kb)
     assert (mask_g == 1).all()
+
+
+@pytest.mark.parametrize("name,kw", [("tiny", {}), ("wan1p3b_480p", dict(H=3, T=5)), ("cogvideox5b", dict(H=5, T=3)),
+                                     ("hunyuan_720p", dict(H=2, T=2)), ("wan14b_720p", dict(H=3)), ("hunyuan_720p", dict(H=2))])
+def test_fused_kernel_and_three_kernel_path_agree(name, kw):
+    """Top-k mode normally runs as one persistent kernel that pools on the tensor cores; the three separate kernels pool
+    with CUDA-core sums.  The pooled scores may differ in the last bits (order of the fp32 sums), far inside the 2e-5
+    the oracle comparison allows; masks may differ only where a score sits that close to the row's threshold."""
+    w = wl.shrunk(wl.get(name), **kw) if kw else wl.get(name)
+    nthreads = min(16, os.cpu_count() or 1)
+    Q = to_dev(wl.gen_tensor(w, "Q", "history", threads=nthreads))
+    K = to_dev(wl.gen_tensor(w, "K", "history", threads=nthreads))
+    shape = cn.shape_of(w, Q, K)
+    out = []
+    try:
+        for path in (cn.BUILDER_FUSED, cn.BUILDER_THREE_KERNELS):
+            cn.debug_set_builder_path(path)
+            scores = torch.full((w.B, w.H, w.nqb, w.nkb), float("nan"), dtype=torch.float32, device="cuda")
+            mask, ws = cn.build_connectivity(Q, K, shape, cn.params_of(w.build), pooled_scores=scores)
+            assert cn.query_status(ws) == cn.OK, cn.last_cuda_error()
+            mask2, ws = cn.build_connectivity(Q, K, shape, cn.params_of(w.build), ws=ws)       # without the score output
+            assert cn.query_status(ws) == cn.OK
+            assert torch.equal(mask, mask2)
+            out.append((mask, scores))
+    finally:
+        cn.debug_set_builder_path(cn.BUILDER_AUTO)
+    (m0, s0), (m1, s1) = out
+    assert float((s0 - s1).abs().max()) <= 5e-6
+    assert bool((m0.sum(-1) == m1.sum(-1)).all())                       # top-k: same number of blocks per row
+    assert int((m0 != m1).sum()) <= 1e-5 * m0.numel() + 2
 
 
 # the HunyuanVideo-shaped layer also at the ends of its density sweep
