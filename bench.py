@@ -6,11 +6,16 @@ Q/K pair (pool, score, select), mask compaction, sparse attention.  The headline
 effective TFLOP/s on computed tiles (4 * rows * cols * D per evaluated block pair) over the whole
 step; ms per attention layer is reported beside it.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--density R]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--density R] [--legs LIST]
     python bench.py --impl reference ...      # the CPU oracle on a bounded sample of the same workload
 
-Under torchrun (N > 1) every rank runs an independent replica of the workload on its own GPU
-(the path has no exchange step); times are the max over ranks.
+The same JSON line also carries the other measured claims (`--legs`, default all): `configs` (attention on the
+other workload shapes), `density_sweep` (the HunyuanVideo-shaped layer at its five keep ratios with a least-squares
+ns-per-tile fit), `exact_builder`, `regions`, `seed_expansion`; each leg samples the clocks for itself.
+
+With N > 1 every rank runs an independent replica of the workload on its own GPU (the path has no exchange
+step); times are the max over ranks.  `--gpus N` starts the N ranks by itself unless it already runs under
+torchrun (WORLD_SIZE set).
 """
 from __future__ import annotations
 
@@ -44,10 +49,12 @@ def parse_args():
     ap.add_argument("--density", type=float, default=None, help="override the builder's keep ratio")
     ap.add_argument("--attn-impl", default="auto", choices=["auto", "portable", "tcgen05"])
     ap.add_argument("--heads", type=int, default=None, help="run a slice with fewer heads (profiling captures)")
-    ap.add_argument("--exact-builder", action="store_true",
-                    help="also time carnator_build_connectivity_exact (block masses on the tensor cores) on the history pair")
-    ap.add_argument("--regions", action="store_true",
-                    help="also time the region builder, latent fusion and the region-restricted attention form")
+    ap.add_argument("--legs", default=None,
+                    help="comma list of extra legs: configs,density_sweep,exact_builder,regions,seed_expansion; 'none'; "
+                         "default: all for the default workload with all heads, none otherwise")
+    ap.add_argument("--exact-builder", action="store_true", help="same as adding exact_builder to --legs")
+    ap.add_argument("--regions", action="store_true", help="same as adding regions to --legs")
+    ap.add_argument("--selftest-launch", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=15.0, help="target CPU time of the oracle sample")
@@ -216,6 +223,18 @@ def max_over_ranks(values, device=None):
     return [float(v) for v in t.tolist()]
 
 
+def all_ranks(value, device=None):
+    """Every rank's value, in rank order (a one-element list when not distributed)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return [float(value)]
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    out = [torch.zeros_like(t) for _ in range(dist.get_world_size())]
+    dist.all_gather(out, t)
+    return [float(o.item()) for o in out]
+
+
 def whole_job_tflops(flops_per_replica: float, world: int, ms_per_step: float) -> float:
     """Every rank runs one replica of the workload; the job's throughput is all replicas' work over the slowest rank's time."""
     return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
@@ -224,6 +243,237 @@ def whole_job_tflops(flops_per_replica: float, world: int, ms_per_step: float) -
 # ------------------------------------------------------------------------------------------------
 # GPU arm
 # ------------------------------------------------------------------------------------------------
+ALL_LEGS = ("configs", "density_sweep", "exact_builder", "regions", "seed_expansion")
+N_SM = 148
+MUFU_PER_CLK_SM = 16          # exponentials per clock and SM (measured: 128 x 128 exponentials take 1024 clocks of one SM)
+
+
+def legs_from_args(args):
+    if args.legs is None:
+        legs = set(ALL_LEGS) if (args.workload == "wan14b_720p" and args.heads is None and args.density is None) else set()
+    elif args.legs.strip().lower() in ("none", ""):
+        legs = set()
+    elif args.legs.strip().lower() == "all":
+        legs = set(ALL_LEGS)
+    else:
+        legs = {x.strip() for x in args.legs.split(",") if x.strip()}
+        bad = legs - set(ALL_LEGS)
+        if bad:
+            raise SystemExit(f"unknown legs {sorted(bad)}; choose from {ALL_LEGS}")
+    if args.exact_builder:
+        legs.add("exact_builder")
+    if args.regions:
+        legs.add("regions")
+    return legs
+
+
+def mufu_bound_ms(tiles, block, sm_mhz):
+    """Time the exponential unit alone needs for block x block exponentials per listed tile."""
+    if not sm_mhz:
+        return None
+    return tiles * float(block) * block / (MUFU_PER_CLK_SM * N_SM * sm_mhz * 1e6) * 1e3
+
+
+class Device:
+    """Device-side state shared by the legs: binding, peaks, transfer helper, timing helper."""
+
+    def __init__(self, local, impl, peaks):
+        import torch
+        from paper_2609_32420_b200 import carnator as cn
+        self.torch, self.cn = torch, cn
+        self.local, self.impl, self.peaks = local, impl, peaks
+        self.dev = torch.device("cuda", local)
+
+    def to_dev(self, bits):
+        return self.torch.from_numpy(bits.view(np.int16)).to(self.dev).view(self.torch.bfloat16)
+
+    def timed(self, fn, n, warm=3):
+        """Mean ms of n calls after `warm` untimed ones, CUDA events on the current stream, clocks sampled meanwhile."""
+        torch = self.torch
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(self.local)
+        sampler.start()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
+        ev[0].record()
+        for i in range(n):
+            fn()
+            ev[i + 1].record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        ts = [ev[i].elapsed_time(ev[i + 1]) for i in range(n)]
+        return float(np.mean(ts)), float(np.min(ts)), clocks
+
+
+def attention_leg(D, w, n, inputs=None, keep=None):
+    """Builder on the history pair, compaction and attention of one workload; returns the timings of each and the
+    roofline fractions of the attention kernel.  `inputs` carries device tensors between calls on the same workload."""
+    torch, cn = D.torch, D.cn
+    if keep is not None:
+        w = w.replace(build=dataclasses.replace(w.build, keep_ratio=keep))
+    if inputs is None:
+        inputs = {}
+    if "Q" not in inputs:
+        which = "history" if w.history_mask else "target"
+        for t in "QKV":
+            inputs[t] = D.to_dev(gen_parallel(w, t, "target"))
+        inputs["Qh"] = D.to_dev(gen_parallel(w, "Q", which))
+        inputs["Kh"] = D.to_dev(gen_parallel(w, "K", which))
+        inputs["rec_np"] = wl.gen_recompute_rows(w)
+        inputs["rec"] = torch.from_numpy(inputs["rec_np"]).to(D.dev)
+        inputs["O"] = torch.empty((w.B, w.H, w.N, w.D), dtype=torch.bfloat16, device=D.dev)
+        inputs["LSE"] = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device=D.dev)
+        inputs["mask"] = torch.empty((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=D.dev)
+    Q, K, V, Qh, Kh, O, LSE, mask, rec = (inputs[k] for k in ("Q", "K", "V", "Qh", "Kh", "O", "LSE", "mask", "rec"))
+    shape = cn.shape_of(w, Q, K, V, None, attn_impl=D.impl)
+    shape.o_stride = type(shape.o_stride)(*O.stride()[:3])
+    bshape = cn.shape_of(w, Qh, Kh)
+    params = cn.params_of(w.build)
+    if "bws" not in inputs:
+        inputs["bws"] = torch.empty(cn.build_workspace_bytes(bshape, params), dtype=torch.uint8, device=D.dev)
+        inputs["aws"] = torch.empty(cn.attn_workspace_bytes(shape), dtype=torch.uint8, device=D.dev)
+    bws, aws = inputs["bws"], inputs["aws"]
+    ms_build, _, _ = D.timed(lambda: cn.build_connectivity(Qh, Kh, bshape, params, mask=mask, ws=bws), max(n, 5))
+    ms_compact, _, _ = D.timed(lambda: cn.compact_mask(mask, rec, shape, ws=aws), max(n, 5))
+    tiles = cn.compacted_tiles(shape, aws)
+    ms_attn, ms_min, clocks = D.timed(lambda: cn.sparse_attn_compacted(Q, K, V, shape, aws, O=O, LSE=LSE), n)
+    st = cn.query_status(aws)
+    if st != cn.OK:
+        raise SystemExit(f"{w.name}: device status {st}: {cn.last_cuda_error()}")
+    from_mask = (mask.cpu().numpy() != 0) | (inputs["rec_np"] != 0)[:, None, :, None]
+    rq = np.minimum(w.block, w.N - np.arange(w.nqb) * w.block).astype(np.float64)
+    flops = 4.0 * w.D * float(np.einsum("bhij,i,j->", from_mask.astype(np.float64), rq, rq))
+    tflops = flops / (ms_attn * 1e-3) / 1e12
+    mufu = mufu_bound_ms(tiles, w.block, clocks.get("sm_mhz"))
+    qk_bytes = 2.0 * w.B * w.H * w.N * w.D * 2
+    out = {"workload": w.name, "H": w.H, "N": w.N, "D": w.D, "block": w.block, "keep_ratio": w.build.keep_ratio,
+           "effective_density": float(from_mask.mean()), "computed_tiles": int(tiles), "flops": flops,
+           "ms_attn": ms_attn, "ms_attn_min": ms_min, "ms_compact": ms_compact, "ms_build": ms_build,
+           "attn_tflops": tflops, "frac_of_bf16_burst": tflops / D.peaks["bf16"],
+           "frac_of_bf16_sustained": tflops / D.peaks["bf16_sustained"],
+           "mufu_bound_ms": mufu, "frac_of_mufu_bound": (mufu / ms_attn) if mufu else None,
+           "builder_gbs": qk_bytes / (ms_build * 1e-3) / 1e9, "builder_frac_of_hbm": qk_bytes / (ms_build * 1e-3) / 1e9 / D.peaks["hbm"],
+           "executor": "tcgen05" if (w.block == 128 and D.impl != D.cn.IMPL_PORTABLE) else "portable (mma.sync)",
+           "steps": n, "clocks": clocks}
+    return out, inputs
+
+
+def leg_configs(D, n):
+    """Attention (and builder, compaction) on the other workload shapes; the HunyuanVideo-shaped one is in density_sweep."""
+    out = []
+    for name in ("tiny", "wan1p3b_480p", "cogvideox5b"):
+        r, inputs = attention_leg(D, wl.get(name), n)
+        out.append(r)
+        del inputs
+        D.torch.cuda.empty_cache()
+    return out
+
+
+def leg_density_sweep(D, n):
+    """The HunyuanVideo-shaped layer at its five keep ratios: time against listed tiles, least-squares line."""
+    w = wl.get("hunyuan_720p")
+    inputs, pts = None, []
+    for keep in wl.HUNYUAN_DENSITIES:
+        r, inputs = attention_leg(D, w, n, inputs, keep=keep)
+        pts.append(r)
+    del inputs
+    D.torch.cuda.empty_cache()
+    x = np.array([p["computed_tiles"] for p in pts], dtype=np.float64)
+    y = np.array([p["ms_attn"] for p in pts], dtype=np.float64)
+    slope, intercept = np.polyfit(x, y, 1)
+    resid = y - (slope * x + intercept)
+    return {"workload": w.name, "points": pts, "ns_per_tile": slope * 1e6, "intercept_ms": float(intercept),
+            "max_abs_residual_ms": float(np.abs(resid).max()),
+            "ns_per_tile_at_each_point": [float(v) for v in (y / x * 1e6)]}
+
+
+def leg_exact_builder(D, w, inputs, n):
+    """carnator_build_connectivity_exact on the history pair (second pass over Q K^T with the dense run's LSE).  Every score
+    costs one exponential and D multiply-adds on the tensor cores, so the exponential unit bounds the kernel."""
+    torch, cn = D.torch, D.cn
+    Qh, Kh = inputs["Qh"], inputs["Kh"]
+    bshape = cn.shape_of(w, Qh, Kh)
+    Lh = dense_lse(D, w, inputs)
+    xparams = cn.params_of(dataclasses.replace(w.build, mode=wl.MODE_CUMMASS))
+    xmask = torch.empty((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=D.dev)
+    xws = torch.empty(cn.exact_workspace_bytes(bshape), dtype=torch.uint8, device=D.dev)
+    ms, ms_min, clocks = D.timed(lambda: cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, ws=xws), n)
+    x_flops = 2.0 * w.B * w.H * float(w.N) * float(w.N) * w.D
+    tiles = w.B * w.H * w.nqb * w.nkb
+    mufu = mufu_bound_ms(tiles, w.block, clocks.get("sm_mhz"))
+    tf = x_flops / (ms * 1e-3) / 1e12
+    return {"ms": ms, "ms_min": ms_min, "tflops": tf, "flops_per_launch": x_flops, "mass": w.build.mass,
+            "density": float(xmask.float().mean()), "status": cn.query_status(xws), "steps": n,
+            "bound": "exponential unit", "mufu_bound_ms": mufu, "frac_of_mufu_bound": (mufu / ms) if mufu else None,
+            "frac_of_bf16_burst": tf / D.peaks["bf16"], "clocks": clocks}
+
+
+def dense_lse(D, w, inputs):
+    """LSE of the history pair under an all-ones mask (shared by the exact builder and the seed expansion legs)."""
+    torch, cn = D.torch, D.cn
+    if "Lh" not in inputs:
+        Qh, Kh = inputs["Qh"], inputs["Kh"]
+        ones = torch.ones((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=D.dev)
+        Vz = torch.zeros_like(Kh)
+        hsh = cn.shape_of(w, Qh, Kh, Vz, None, attn_impl=D.impl)
+        _, inputs["Lh"], _ = cn.sparse_attn(Qh, Kh, Vz, ones, None, hsh)
+        del Vz, ones
+    return inputs["Lh"]
+
+
+def leg_seed_expansion(D, w, inputs, n):
+    """carnator_seed_expansion: reads Q once (the seed keys are a few hundred rows), so HBM bandwidth bounds it."""
+    torch, cn = D.torch, D.cn
+    Qh, Kh = inputs["Qh"], inputs["Kh"]
+    Lh = dense_lse(D, w, inputs)
+    rng = np.random.default_rng(5)
+    n_pos, n_neg = 192, 320
+    tok = rng.choice(np.arange(w.n_text, w.N), size=n_pos + n_neg, replace=False).astype(np.int32)
+    seeds = torch.from_numpy(tok).to(D.dev)
+    shape = cn.shape_of(w, Qh, Kh)
+    ms, ms_min, clocks = D.timed(lambda: cn.seed_expansion(Qh, Kh, Lh, seeds, n_pos, n_neg, shape), n)
+    nbytes = float(w.B) * w.H * w.N * (w.D * 2 + 4 + 4) + float(w.B) * w.N * 4     # Q, LSE, per-head contrast, result
+    return {"ms": ms, "ms_min": ms_min, "n_pos": n_pos, "n_neg": n_neg, "bound": "hbm", "bytes_per_launch": nbytes,
+            "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm": nbytes / (ms * 1e-3) / 1e9 / D.peaks["hbm"],
+            "executor": "mma.sync (Q x K_seed^T on gathered key rows)", "steps": n, "clocks": clocks,
+            "note": "includes the allocation of its workspace and output by the binding"}
+
+
+def leg_regions(D, w, inputs, n):
+    """Region builder, latent fusion and the region-restricted attention form on the workload's grid."""
+    torch, cn = D.torch, D.cn
+    Q, K, V, O, LSE, mask = (inputs[k] for k in ("Q", "K", "V", "O", "LSE", "mask"))
+    shape = cn.shape_of(w, Q, K, V, None, attn_impl=D.impl)
+    shape.o_stride = type(shape.o_stride)(*O.stride()[:3])
+    rng = np.random.default_rng(77)
+    ev = np.zeros((w.T, w.Hg, w.Wg), dtype=np.uint8)
+    cy, cx = w.Hg // 2, w.Wg // 2
+    for t in range(w.T):                                   # one drifting object tube, about 6 % of each frame
+        cy = int(np.clip(cy + rng.integers(-1, 2), 6, w.Hg - 7)); cx = int(np.clip(cx + rng.integers(-2, 3), 10, w.Wg - 11))
+        ev[t, cy - 5:cy + 6, cx - 9:cx + 10] = 1
+    evd = torch.from_numpy(ev).to(D.dev)
+    ms_regions, _, _ = D.timed(lambda: cn.build_regions(evd, shape, 2, 3), 20)
+    act, ctx, Wt = cn.build_regions(evd, shape, 2, 3)
+    C_lat = 64                                             # latent channels per token (16 x 2 x 2 patch)
+    zt = torch.randn((C_lat, w.T * w.Hg * w.Wg), dtype=torch.float32, device=D.dev)
+    zh = torch.randn_like(zt); zo = torch.empty_like(zt)
+    Wf = Wt.reshape(-1)
+    ms_fuse, _, _ = D.timed(lambda: cn.fuse_latents(zt, zh, Wf, z_out=zo), 20)
+    fuse_bytes = 3.0 * zt.numel() * 4 + Wt.numel() * 4
+    aq = cn.region_block_flags(act, shape, w.block, 1).reshape(1, -1).contiguous()
+    ck = cn.region_block_flags(ctx, shape, w.block, 1).reshape(1, -1).contiguous()
+    rws = torch.empty(cn.attn_workspace_bytes(shape), dtype=torch.uint8, device=D.dev)
+    ms_rattn, _, clocks = D.timed(lambda: cn.sparse_attn_region(Q, K, V, mask, aq, ck, shape, O, LSE, ws=rws), n)
+    rtiles = cn.compacted_tiles(shape, rws)
+    rt = rtiles * 4.0 * w.block * w.block * w.D / (ms_rattn * 1e-3) / 1e12
+    return {"ms_build_regions": ms_regions, "ms_fuse_latents": ms_fuse, "fuse_bound": "hbm",
+            "fuse_gbs": fuse_bytes / (ms_fuse * 1e-3) / 1e9, "fuse_frac_of_hbm": fuse_bytes / (ms_fuse * 1e-3) / 1e9 / D.peaks["hbm"],
+            "active_query_blocks": int(aq.sum()), "context_key_blocks": int(ck.sum()),
+            "ms_region_attn": ms_rattn, "region_tiles": rtiles, "region_attn_bound": "tensor",
+            "region_attn_tflops": rt, "region_attn_frac_of_bf16_burst": rt / D.peaks["bf16"], "clocks": clocks}
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -233,8 +483,19 @@ def run_ours(args):
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.selftest_launch:                     # CPU check of the launch path: gloo ranks, a stand-in step
+        dist.init_process_group("gloo")
+        ms = max_over_ranks([10.0 + 5.0 * rank])
+        per_rank = all_ranks(10.0 + 5.0 * rank)
+        if rank == 0:
+            print(json.dumps({"selftest": True, "n_gpus": world, "ms_per_step": ms[0], "ms_per_rank": per_rank,
+                              "config": {"parallelism": "replicas only"}}), flush=True)
+        dist.destroy_process_group()
+        return
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    if local >= torch.cuda.device_count():
+        raise SystemExit(f"rank {rank}: no GPU {local} on this machine ({torch.cuda.device_count()} visible)")
     torch.cuda.set_device(local)
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
@@ -247,10 +508,10 @@ def run_ours(args):
     w = workload_from_args(args)
     impl = {"auto": cn.IMPL_AUTO, "portable": cn.IMPL_PORTABLE, "tcgen05": cn.IMPL_TCGEN05}[args.attn_impl]
     peaks = load_peaks()
-    dev = torch.device("cuda", local)
-
-    def to_dev(bits):
-        return torch.from_numpy(bits.view(np.int16)).to(dev).view(torch.bfloat16)
+    legs = legs_from_args(args)
+    D = Device(local, impl, peaks)
+    dev = D.dev
+    to_dev = D.to_dev
 
     which = "history" if w.history_mask else "target"
     host = {}
@@ -317,77 +578,18 @@ def run_ours(args):
     ms_compact = float(np.mean([e[1].elapsed_time(e[2]) for e in evs]))
     ms_attn = float(np.mean([e[2].elapsed_time(e[3]) for e in evs]))
     ms_attn_min = float(np.min([e[2].elapsed_time(e[3]) for e in evs]))
+    ms_per_rank = all_ranks(total_ms / args.steps, dev)
     total_ms, ms_attn = max_over_ranks([total_ms, ms_attn], dev)
     ms_step = total_ms / args.steps
     value = whole_job_tflops(flops, world, ms_step)
 
-    # ---- optional: the exact block-mass builder (second pass over Q K^T with the dense run's LSE) --------
-    exact = None
-    if args.exact_builder:
-        ones = torch.ones((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=dev)
-        Vz = torch.zeros_like(Kh)
-        hsh = cn.shape_of(w, Qh, Kh, Vz, None, attn_impl=impl)
-        _, Lh, _ = cn.sparse_attn(Qh, Kh, Vz, ones, None, hsh)
-        del Vz, ones
-        xparams = cn.params_of(dataclasses.replace(w.build, mode=wl.MODE_CUMMASS))
-        xmask = torch.empty((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device=dev)
-        xws = torch.empty(cn.exact_workspace_bytes(bshape), dtype=torch.uint8, device=dev)
-        for _ in range(3):
-            cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, ws=xws)
-        torch.cuda.synchronize()
-        n_x = max(3, min(args.steps, 10))
-        xe = [torch.cuda.Event(enable_timing=True) for _ in range(n_x + 1)]
-        xe[0].record()
-        for i in range(n_x):
-            cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, ws=xws)
-            xe[i + 1].record()
-        torch.cuda.synchronize()
-        x_ms = float(np.mean([xe[i].elapsed_time(xe[i + 1]) for i in range(n_x)]))
-        x_flops = 2.0 * w.B * w.H * float(w.N) * float(w.N) * w.D
-        exact = {"ms": x_ms, "tflops": x_flops / (x_ms * 1e-3) / 1e12, "frac": x_flops / (x_ms * 1e-3) / 1e12 / peaks["bf16"],
-                 "flops_per_launch": x_flops, "mass": w.build.mass, "density": float(xmask.float().mean()),
-                 "status": cn.query_status(xws), "steps": n_x, "bound": "tensor", "peak": peaks["bf16"]}
-        del Lh, xmask, xws
-
-    # ---- optional: reuse regions, latent fusion, region-restricted attention ---------------------------------
-    regions = None
-    if args.regions:
-        rng = np.random.default_rng(77)
-        ev = np.zeros((w.T, w.Hg, w.Wg), dtype=np.uint8)
-        cy, cx = w.Hg // 2, w.Wg // 2
-        for t in range(w.T):                                   # one drifting object tube, about 6 % of each frame
-            cy = int(np.clip(cy + rng.integers(-1, 2), 6, w.Hg - 7)); cx = int(np.clip(cx + rng.integers(-2, 3), 10, w.Wg - 11))
-            ev[t, cy - 5:cy + 6, cx - 9:cx + 10] = 1
-        evd = torch.from_numpy(ev).to(dev)
-
-        def timed(fn, n=20):
-            for _ in range(3):
-                fn()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            torch.cuda.synchronize(); e0.record()
-            for _ in range(n):
-                fn()
-            e1.record(); torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / n
-
-        ms_regions = timed(lambda: cn.build_regions(evd, shape, 2, 3))
-        act, ctx, Wt = cn.build_regions(evd, shape, 2, 3)
-        C_lat = 64                                             # latent channels per token (16 x 2 x 2 patch)
-        zt = torch.randn((C_lat, w.T * w.Hg * w.Wg), dtype=torch.float32, device=dev)
-        zh = torch.randn_like(zt); zo = torch.empty_like(zt)
-        ms_fuse = timed(lambda: cn.fuse_latents(zt, zh, Wt.reshape(-1), z_out=zo))
-        fuse_bytes = 3.0 * zt.numel() * 4 + Wt.numel() * 4
-        aq = cn.region_block_flags(act, shape, w.block, 1).reshape(1, -1).contiguous()
-        ck = cn.region_block_flags(ctx, shape, w.block, 1).reshape(1, -1).contiguous()
-        rws = torch.empty(cn.attn_workspace_bytes(shape), dtype=torch.uint8, device=dev)
-        ms_rattn = timed(lambda: cn.sparse_attn_region(Q, K, V, mask, aq, ck, shape, O, LSE, ws=rws), n=5)
-        rtiles = cn.compacted_tiles(shape, rws)
-        regions = {"ms_build_regions": ms_regions, "ms_fuse_latents": ms_fuse,
-                   "fuse_gbs": fuse_bytes / (ms_fuse * 1e-3) / 1e9, "fuse_frac_of_hbm": fuse_bytes / (ms_fuse * 1e-3) / 1e9 / peaks["hbm"],
-                   "active_query_blocks": int(aq.sum()), "context_key_blocks": int(ck.sum()),
-                   "ms_region_attn": ms_rattn, "region_tiles": rtiles,
-                   "region_attn_tflops": rtiles * 4.0 * w.block * w.block * w.D / (ms_rattn * 1e-3) / 1e12}
-        del zt, zh, zo, rws
+    # ---- extra legs that work on the headline workload's resident tensors (rank 0 reports them) -------------
+    inputs = {"Q": Q, "K": K, "V": V, "Qh": Qh, "Kh": Kh, "O": O, "LSE": LSE, "mask": mask}
+    n_leg = max(3, min(args.steps, 6))
+    exact = leg_exact_builder(D, w, inputs, n_leg) if "exact_builder" in legs else None
+    seed = leg_seed_expansion(D, w, inputs, n_leg) if "seed_expansion" in legs else None
+    inputs.pop("Lh", None)
+    regions = leg_regions(D, w, inputs, n_leg) if "regions" in legs else None
 
     # ---- end to end through the host-buffer calls --------------------------------------------------
     e2e = None
@@ -400,6 +602,7 @@ def run_ours(args):
         hO = torch.empty((w.B, w.H, w.N, w.D), dtype=torch.int16).pin_memory()
         hL = torch.empty((w.B, w.H, w.N), dtype=torch.float32).pin_memory()
         del Qh, Kh
+        inputs.pop("Qh"); inputs.pop("Kh")
         arena = torch.empty(max(cn.attn_host_arena_bytes(hshape), cn.build_host_arena_bytes(hshape, params)),
                             dtype=torch.uint8, device=dev)
 
@@ -425,26 +628,37 @@ def run_ours(args):
                "note": "carnator_build_connectivity_host + carnator_sparse_attn_host, pinned host buffers"}
         same = bool((hmask.numpy() == mask_np).all())
         e2e["mask_equals_device_run"] = same
+        del arena, pin, hO, hL, hmask
 
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
+    # ---- legs on other workloads: release the headline tensors first ---------------------------------
+    del Q, K, V, O, LSE, mask, inputs, bws, aws
+    host.clear()
+    torch.cuda.empty_cache()
+    configs = leg_configs(D, n_leg) if "configs" in legs else None
+    sweep = leg_density_sweep(D, n_leg) if "density_sweep" in legs else None
+
     # ---- roofline of the dominant kernel -----------------------------------------------------------
     attn_tflops = flops / (ms_attn * 1e-3) / 1e12
-    traffic = None
+    traffic, traffic_src = None, None
     tpath = os.path.join(ROOT, "profiles", "attn_traffic.txt")
     if os.path.exists(tpath):
         base = w.name.split("[")[0]
         for ln in open(tpath):
             parts = ln.split()
-            if len(parts) == 3 and parts[0] == base and int(parts[2]) > 0:
+            if len(parts) >= 3 and parts[0] == base and int(parts[2]) > 0:
                 traffic = float(parts[1]) * tiles / float(parts[2])
+                traffic_src = "profiles/attn_traffic.txt" + (f" (captured at {parts[3]})" if len(parts) > 3 else "")
+    mufu = mufu_bound_ms(tiles, w.block, clocks.get("sm_mhz"))
     roofline = {"bound": "tensor", "kernel": "sparse attention", "achieved": attn_tflops, "peak": peaks["bf16"],
-                "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16"], "traffic": traffic,
+                "unit": "TFLOP/s", "frac": attn_tflops / peaks["bf16"], "traffic": traffic, "traffic_source": traffic_src,
                 "peak_source": peaks["source"] + " bf16_tflops (burst)", "frac_of_sustained": attn_tflops / peaks["bf16_sustained"],
-                "frac_of_nominal_2250": attn_tflops / 2250.0, "flops_per_launch": flops}
+                "frac_of_nominal_2250": attn_tflops / 2250.0, "flops_per_launch": flops,
+                "mufu_bound_ms": mufu, "frac_of_mufu_bound": (mufu / ms_attn) if mufu else None}
     qk_bytes = 2.0 * w.B * w.H * w.N * w.D * 2
     builder = {"bound": "hbm", "ms": ms_build, "achieved": qk_bytes / (ms_build * 1e-3) / 1e9, "peak": peaks["hbm"],
                "unit": "GB/s", "frac": qk_bytes / (ms_build * 1e-3) / 1e9 / peaks["hbm"], "bytes_per_launch": qk_bytes}
@@ -462,22 +676,68 @@ def run_ours(args):
                    "keep_ratio": w.build.keep_ratio, "effective_density": density, "computed_tiles": tiles,
                    "l2": "inputs larger than L2 (no flush needed)", "attn_impl": args.attn_impl,
                    "parallelism": "replicas only" if world > 1 else "single GPU"},
+        "ms_per_rank": ms_per_rank,
         "ms_attn_layer": ms_attn, "ms_attn_layer_min": ms_attn_min, "ms_compact": ms_compact, "ms_build": ms_build,
         "attn_tflops": attn_tflops, "clocks": clocks, "gpu_launches": int(launches),
         "roofline": roofline, "builder_roofline": builder, "cpu_baseline": cpu, "e2e": e2e,
     }
+    if configs is not None:
+        line["configs"] = configs
+    if sweep is not None:
+        line["density_sweep"] = sweep
     if exact is not None:
         line["exact_builder"] = exact
     if regions is not None:
         line["regions"] = regions
+    if seed is not None:
+        line["seed_expansion"] = seed
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------------
+# --gpus N without torchrun: start the N replicas here
+# ------------------------------------------------------------------------------------------------
+def free_port() -> int:
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
+def launch_replicas(args) -> int:
+    """Re-runs this command line as N ranks (one GPU each, rendezvous on 127.0.0.1) and passes rank 0's line through.
+    The ranks are independent replicas; torch.distributed only carries the MAX of their timings."""
+    n = args.gpus
+    if not args.selftest_launch and args.impl == "ours":
+        import torch
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < n:
+            sys.stderr.write(f"bench.py --gpus {n}: this machine shows {have} GPU(s); refusing to report fewer replicas than asked for\n")
+            return 2
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
+                                      stdout=subprocess.PIPE if r == 0 else subprocess.DEVNULL, text=True))
+    out, _ = procs[0].communicate()
+    rc = procs[0].returncode
+    for p in procs[1:]:
+        p.wait()
+        rc = rc or p.returncode
+    sys.stdout.write(out)
+    sys.stdout.flush()
+    return rc
+
+
 def main():
     args = parse_args()
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and (args.impl == "ours" or args.selftest_launch):
+        raise SystemExit(launch_replicas(args))
+    if args.impl == "reference" and not args.selftest_launch:
         run_reference(args)
     else:
         run_ours(args)

@@ -68,3 +68,37 @@ def test_reference_arm_prints_one_json_line():
     out1 = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "tiny",
                            "--steps", "1", "--warmup", "0"], capture_output=True, text=True, env=dict(os.environ, RANK="1"), timeout=60)
     assert out1.returncode == 0 and out1.stdout.strip() == ""
+
+
+def test_gpus_flag_starts_the_ranks_itself_gloo_world2():
+    """`bench.py --gpus 2` without torchrun: the launcher starts two ranks (rendezvous on 127.0.0.1); here they are gloo ranks
+    on CPU running a stand-in step, and rank 0's line must report both."""
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--selftest-launch"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert out.returncode == 0, out.stderr
+    line = json.loads(out.stdout.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["ms_per_rank"] == [10.0, 15.0] and line["ms_per_step"] == 15.0
+    assert line["config"]["parallelism"] == "replicas only"
+
+
+def test_gpus_flag_fails_loudly_when_the_machine_has_fewer_gpus():
+    import torch
+    have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")}
+    out = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", str(max(have, 1) + 1), "--steps", "1"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert out.returncode != 0 and out.stdout.strip() == ""
+    assert "refusing to report fewer replicas" in out.stderr
+
+
+def test_leg_selection():
+    ns = lambda **kw: type("A", (), dict(dict(legs=None, workload="wan14b_720p", heads=None, density=None,
+                                               exact_builder=False, regions=False), **kw))()
+    assert bench.legs_from_args(ns()) == set(bench.ALL_LEGS)                    # default run carries every leg
+    assert bench.legs_from_args(ns(heads=4)) == set()                           # profiling slices stay lean
+    assert bench.legs_from_args(ns(legs="none", regions=True)) == {"regions"}
+    assert bench.legs_from_args(ns(legs="configs,density_sweep")) == {"configs", "density_sweep"}
+    with pytest.raises(SystemExit):
+        bench.legs_from_args(ns(legs="bogus"))
+    assert bench.mufu_bound_ms(148 * 16, 128, 1000.0) == pytest.approx(16 * 1024 / 1e9 * 1e3)   # 16 tiles per SM, 1024 clocks each
