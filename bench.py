@@ -86,38 +86,65 @@ def gen_parallel(w, tensor, which):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons with nvidia-smi while a timed region runs.
+
+    One nvidia-smi process per GPU serves the whole run (its start-up takes longer than a short leg); every line is
+    stamped with the host clock when it arrives, and a region takes the samples that fall between its start() and
+    stop().  A region shorter than the sampling period takes the sample nearest to it and says so."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    PERIOD_MS = 25
+    _shared = {}            # GPU index -> (process, list of (host time, line))
 
     def __init__(self, index: int):
         self.index = index
         self.proc = None
         self.lines = []
+        self.t0 = None
+
+    @classmethod
+    def _feed(cls, index):
+        if index in cls._shared:
+            return cls._shared[index]
+        try:
+            proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={cls.FIELDS}", "--format=csv,noheader,nounits", "-lms", str(cls.PERIOD_MS),
+                 "-i", str(index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            cls._shared[index] = (None, [])
+            return cls._shared[index]
+        log = []
+
+        def read():
+            for line in proc.stdout:
+                log.append((time.perf_counter(), line.strip()))
+        threading.Thread(target=read, daemon=True).start()
+        import atexit
+        atexit.register(proc.terminate)
+        cls._shared[index] = (proc, log)
+        return cls._shared[index]
 
     def start(self):
-        try:
-            self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "25",
-                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
-            self.thread.start()
-        except Exception:
-            self.proc = None
-
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+        self.proc, self._log = self._feed(self.index)
+        self.t0 = time.perf_counter()
 
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except Exception:
-            self.proc.kill()
+        t1 = time.perf_counter()
+        if self.t0 is not None:
+            inside = [ln for (t, ln) in list(self._log) if self.t0 <= t <= t1 + 1e-3 * self.PERIOD_MS]
+            how = "during"
+            if not inside:              # region shorter than the sampling period: wait for the next sample
+                deadline = time.perf_counter() + 0.5
+                while time.perf_counter() < deadline and not any(t >= self.t0 for (t, _) in list(self._log)):
+                    time.sleep(0.005)
+                later = [ln for (t, ln) in list(self._log) if t >= self.t0]
+                inside, how = later[:1], "first sample after the region"
+            self.lines = inside
+        else:
+            how = "given"
         sm, mx, reasons, power = [], [], set(), []
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in self.lines:
@@ -132,7 +159,8 @@ class ClockSampler:
                 if v.lower().startswith("active"):
                     reasons.add(n)
         return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "power_w_max": max(power) if power else None, "samples": len(sm), "reasons": sorted(reasons)}
+                "power_w_max": max(power) if power else None, "samples": len(sm), "sampled": how,
+                "reasons": sorted(reasons)}
 
 
 # ------------------------------------------------------------------------------------------------
@@ -293,6 +321,11 @@ class Device:
         for _ in range(warm):
             fn()
         torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        fn()
+        torch.cuda.synchronize()
+        once = max(time.perf_counter() - t0, 1e-6)
+        n = int(min(2000, max(n, np.ceil(0.1 / once))))        # at least 0.1 s under load, so that the clocks are sampled
         sampler = ClockSampler(self.local)
         sampler.start()
         ev = [torch.cuda.Event(enable_timing=True) for _ in range(n + 1)]
@@ -355,7 +388,7 @@ def attention_leg(D, w, n, inputs=None, keep=None):
            "mufu_bound_ms": mufu, "frac_of_mufu_bound": (mufu / ms_attn) if mufu else None,
            "builder_gbs": qk_bytes / (ms_build * 1e-3) / 1e9, "builder_frac_of_hbm": qk_bytes / (ms_build * 1e-3) / 1e9 / D.peaks["hbm"],
            "executor": "tcgen05" if (w.block == 128 and D.impl != D.cn.IMPL_PORTABLE) else "portable (mma.sync)",
-           "steps": n, "clocks": clocks}
+           "clocks": clocks}
     return out, inputs
 
 
@@ -404,7 +437,7 @@ def leg_exact_builder(D, w, inputs, n):
     mufu = mufu_bound_ms(tiles, w.block, clocks.get("sm_mhz"))
     tf = x_flops / (ms * 1e-3) / 1e12
     return {"ms": ms, "ms_min": ms_min, "tflops": tf, "flops_per_launch": x_flops, "mass": w.build.mass,
-            "density": float(xmask.float().mean()), "status": cn.query_status(xws), "steps": n,
+            "density": float(xmask.float().mean()), "status": cn.query_status(xws),
             "bound": "exponential unit", "mufu_bound_ms": mufu, "frac_of_mufu_bound": (mufu / ms) if mufu else None,
             "frac_of_bf16_burst": tf / D.peaks["bf16"], "clocks": clocks}
 
@@ -434,9 +467,12 @@ def leg_seed_expansion(D, w, inputs, n):
     shape = cn.shape_of(w, Qh, Kh)
     ms, ms_min, clocks = D.timed(lambda: cn.seed_expansion(Qh, Kh, Lh, seeds, n_pos, n_neg, shape), n)
     nbytes = float(w.B) * w.H * w.N * (w.D * 2 + 4 + 4) + float(w.B) * w.N * 4     # Q, LSE, per-head contrast, result
-    return {"ms": ms, "ms_min": ms_min, "n_pos": n_pos, "n_neg": n_neg, "bound": "hbm", "bytes_per_launch": nbytes,
+    flops = 2.0 * w.B * w.H * w.N * (n_pos + n_neg) * w.D                          # Q x K_seed^T
+    return {"ms": ms, "ms_min": ms_min, "n_pos": n_pos, "n_neg": n_neg, "bytes_per_launch": nbytes, "flops_per_launch": flops,
             "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm": nbytes / (ms * 1e-3) / 1e9 / D.peaks["hbm"],
-            "executor": "mma.sync (Q x K_seed^T on gathered key rows)", "steps": n, "clocks": clocks,
+            "tflops": flops / (ms * 1e-3) / 1e12, "frac_of_bf16_burst": flops / (ms * 1e-3) / 1e12 / D.peaks["bf16"],
+            "bound": "tensor (mma.sync) at this seed count; hbm (read Q once) below about 100 seeds",
+            "executor": "mma.sync (Q x K_seed^T on gathered key rows)", "clocks": clocks,
             "note": "includes the allocation of its workspace and output by the binding"}
 
 
@@ -497,6 +533,7 @@ def run_ours(args):
     if local >= torch.cuda.device_count():
         raise SystemExit(f"rank {rank}: no GPU {local} on this machine ({torch.cuda.device_count()} visible)")
     torch.cuda.set_device(local)
+    ClockSampler._feed(local)                    # nvidia-smi takes a moment to start: long before the first timed region
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     if rank == 0 or world == 1:

@@ -386,6 +386,15 @@ carnator_status carnator_static_status(void* stream);
  * the calling process so far (monotone counter).
  * ------------------------------------------------------------------------ */
 carnator_status carnator_query_status(void* ws, void* stream);
+/* Every wait inside a kernel of this library is bounded: after 2 s (less if the first 256 bytes of the workspace, the
+ * header, carry a shorter wait_limit_ns at byte offset 40 -- written by tests only, the calls that take a workspace
+ * reset it to 0 = default) the waiting role records CARNATOR_ERR_DEVICE_TIMEOUT, the CTA drains what it has in
+ * flight, frees its tensor memory and returns; the device stays usable.
+ * carnator_selftest_wait_timeout runs the wait helper on a barrier that is never armed (one warp, `limit_ns` between
+ * 1 and 2e9): carnator_query_status(ws) must then report CARNATOR_ERR_DEVICE_TIMEOUT.  ws: device, >= 256 bytes,
+ * 256-byte aligned. */
+carnator_status carnator_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream);
+
 /* Testing aid: which path carnator_build_connectivity takes in top-k mode.  0 = by size (the default), 1 = always
  * the three separate kernels (pool, score, select), 2 = the persistent fused kernel wherever it supports the shape.
  * Both compute the same pooled scores up to the order of the fp32 sums.  Process-wide. */

@@ -33,7 +33,7 @@ EXPORTS = [
     "carnator_seed_workspace_bytes", "carnator_seed_expansion",
     "carnator_delta_e00", "carnator_context_discrepancy", "carnator_size_discrepancy", "carnator_shape_discrepancy",
     "carnator_compatibility_gate", "carnator_clopper_pearson_upper",
-    "carnator_query_status", "carnator_debug_set_builder_path", "carnator_status_string", "carnator_last_cuda_error",
+    "carnator_query_status", "carnator_selftest_wait_timeout", "carnator_debug_set_builder_path", "carnator_status_string", "carnator_last_cuda_error",
     "carnator_kernel_launches", "carnator_version",
 ]
 
@@ -151,6 +151,8 @@ def lib() -> ctypes.CDLL:
     L.carnator_clopper_pearson_upper.argtypes = [ctypes.c_int32, ctypes.c_int32, dbl]
     L.carnator_query_status.restype = ctypes.c_int
     L.carnator_query_status.argtypes = [vp, vp]
+    L.carnator_selftest_wait_timeout.restype = ctypes.c_int
+    L.carnator_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint64, vp]
     L.carnator_debug_set_builder_path.restype = None
     L.carnator_debug_set_builder_path.argtypes = [ctypes.c_int32]
     L.carnator_status_string.restype = ctypes.c_char_p
@@ -325,6 +327,14 @@ def compacted_tiles(shape: Shape, ws, stream=None) -> int:
 def query_status(ws, stream=None) -> int:
     return int(lib().carnator_query_status(_ptr(ws), _stream(stream)))
 
+
+def selftest_wait_timeout(ws, limit_ns: int, stream=None) -> None:
+    """carnator_selftest_wait_timeout: a bounded wait on a barrier nothing arms; query_status(ws) reports the time-out."""
+    _check(lib().carnator_selftest_wait_timeout(_ptr(ws), int(limit_ns), _stream(stream)), "carnator_selftest_wait_timeout")
+
+
+# byte offsets inside the 256-byte workspace header (tests of the time-out path write them)
+HDR_WAIT_LIMIT_NS, HDR_DEBUG_WITHHOLD = 40, 48
 
 BUILDER_AUTO, BUILDER_THREE_KERNELS, BUILDER_FUSED = 0, 1, 2
 

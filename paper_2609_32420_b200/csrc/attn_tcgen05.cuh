@@ -85,8 +85,9 @@ __device__ __forceinline__ unsigned long long global_ns() {
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait: gives up after ~2 s (or when another role has aborted) and raises the abort flag.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0) {
+// Bounded wait: gives up after limit_ns (or when another role has aborted) and raises the abort flag.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0,
+                                          unsigned long long limit_ns = kDefaultWaitNs) {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 0; it < (1u << 30); ++it) {
@@ -94,7 +95,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try(bar, parity)) return true;
         if ((it & 255u) == 255u) {
             if (*abort_flag) return false;
-            if (global_ns() - t0 > 2000000000ull) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;
@@ -103,13 +104,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 // Wait used on the way out, after an abort: the copies or products this role still has in flight must land before
 // the CTA gives its shared and tensor memory back, so the abort flag does not end this wait; only time does.
-__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity, unsigned long long limit_ns = kDefaultWaitNs) {
     if (mbar_try(bar, parity)) return true;
     const unsigned long long t0 = global_ns();
     for (uint32_t it = 0; it < (1u << 30); ++it) {
         __nanosleep(100);
         if (mbar_try(bar, parity)) return true;
-        if ((it & 255u) == 255u && global_ns() - t0 > 2000000000ull) break;
+        if ((it & 255u) == 255u && global_ns() - t0 > limit_ns) break;
     }
     return false;
 }
@@ -117,8 +118,9 @@ __device__ __forceinline__ bool mbar_wait_drain(uint32_t bar, uint32_t parity) {
 // Warp-collective form.  Every lane tests the barrier (one broadcast read of shared memory, no divergence in the
 // common case that the phase is already complete); lanes that find it incomplete fall into the bounded wait.  The
 // vote makes the outcome uniform, reconverges the warp and orders the other lanes' later reads after the acquire.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0) {
-    const bool ok = mbar_try(bar, parity) ? true : mbar_wait(bar, parity, abort_flag, sleep_ns);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int* abort_flag, unsigned sleep_ns = 0,
+                                               unsigned long long limit_ns = kDefaultWaitNs) {
+    const bool ok = mbar_try(bar, parity) ? true : mbar_wait(bar, parity, abort_flag, sleep_ns, limit_ns);
     return __all_sync(0xffffffffu, ok) != 0;
 }
 // One arrival per warp once every lane's earlier writes are ordered before it.
@@ -332,6 +334,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
     auto bar_fin = [&](int q) { return bars + 320 + 8 * q; };
     auto bar_pvdone = [&](int s) { return bars + 352 + 8 * s; };     // P V of the step that used score buffer s has completed
     volatile int* abortp = &abort_flag;
+    // every bounded wait of this CTA gives up after `limit` (2 s unless the workspace header asks for less)
+    const unsigned long long limit = a.hdr->wait_limit_ns ? a.hdr->wait_limit_ns : kDefaultWaitNs;
 
     if (tid == 0) {
         abort_flag = 0;
@@ -370,13 +374,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             int armed = -1;
             for (int i = 0; i < T; ++i) {
                 const int s = i % kStages, u = i - kStages;     // the slot is free once Q K^T of step u has completed
-                if (u >= 0 && !mbar_wait(bar_sfull(u & 1), uint32_t(u >> 1) & 1u, abortp, 100)) {
+                if (u >= 0 && !mbar_wait(bar_sfull(u & 1), uint32_t(u >> 1) & 1u, abortp, 100, limit)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 1, i, blockIdx.x); break;
                 }
                 const int J = list[i];
                 if (J < 0 || J >= a.nkb || (i > 0 && J <= list[i - 1])) {      // malformed list: stop before touching memory
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_CHECK, 21, i, blockIdx.x); *abortp = 1; break;
                 }
+                // Test of the time-out path only: the first K tile of the first query block in the order is never
+                // requested, so the wait for it runs out and the CTA takes the abort-and-drain path.
+                if (i == 0 && a.hdr->debug_withhold != 0 && blockIdx.x == 0 && bh == 0) continue;
                 mbar_expect_tx(bar_kfull(s), C::kTileBytes);
                 const int key0 = J * kBlock;
 #pragma unroll
@@ -386,7 +393,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             }
             if (*abortp) {      // copies in flight must land before the CTA gives its shared memory back
                 for (int k = 0; k < kStages && armed - k >= 0; ++k)
-                    mbar_wait_drain(bar_kfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u);
+                    mbar_wait_drain(bar_kfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, limit);
             }
         }
     } else if (warp == kWarpTmaV) {
@@ -395,7 +402,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             int armed = -1;
             for (int i = 0; i < T; ++i) {
                 const int s = i % kStages, u = i - kStages;     // the slot is free once P V of step u has completed
-                if (u >= 0 && !mbar_wait(bar_pvdone(u & 1), uint32_t(u >> 1) & 1u, abortp, 100)) {
+                if (u >= 0 && !mbar_wait(bar_pvdone(u & 1), uint32_t(u >> 1) & 1u, abortp, 100, limit)) {
                     set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 2, i, blockIdx.x); break;
                 }
                 const int J = list[i];
@@ -409,7 +416,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             }
             if (*abortp) {
                 for (int k = 0; k < kStages && armed - k >= 0; ++k)
-                    mbar_wait_drain(bar_vfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u);
+                    mbar_wait_drain(bar_vfull((armed - k) % kStages), uint32_t((armed - k) / kStages) & 1u, limit);
             }
         }
     } else if (warp == kWarpMma) {
@@ -427,7 +434,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             const uint64_t dk = smem_desc(sK, 16, 1024), dv = smem_desc(sV, C::kBoxBytes, 1024);
             const uint32_t k_lo0 = uint32_t(dk), hi_kmajor = uint32_t(dk >> 32);
             const uint32_t v_lo0 = uint32_t(dv), hi_v = uint32_t(dv >> 32);
-            bool ok = mbar_wait_warp(bar_q, 0, abortp);   // the softmax groups have put the query tile into tensor memory
+            bool ok = mbar_wait_warp(bar_q, 0, abortp, 0, limit);   // the softmax groups have put the query tile into tensor memory
             if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 3, 0, blockIdx.x);
             tc_fence_after();
             int iq = 0, ip = 0;                          // next Q K^T step, next P V step
@@ -477,7 +484,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
                         else {
                             const unsigned long long now = global_ns();
                             if (idle == 1024u) t_idle = now;
-                            else if (now - t_idle > 2000000000ull) give_up = 2;
+                            else if (now - t_idle > limit) give_up = 2;
                         }
                     }
                     give_up = __shfl_sync(0xffffffffu, give_up, 0);
@@ -491,7 +498,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             if (ok) tc_commit_el(bar_o);
             if (__any_sync(0xffffffffu, *abortp != 0)) {      // make sure no MMA of this warp is still running before tensor memory is released
                 tc_commit_el(bar_drain);
-                mbar_wait_drain(bar_drain, 0);
+                mbar_wait_drain(bar_drain, 0, limit);
                 __syncwarp();
             }
         }
@@ -543,7 +550,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
         for (int i = wg; i < T; i += 2) {
             const int rs = i % kRefSlots;
             const uint32_t sph = uint32_t(i >> 1) & 1u;
-            ok = mbar_wait_warp(bar_sfull(wg), sph, abortp, 20);   // warp-uniform: the loads below are collective
+            ok = mbar_wait_warp(bar_sfull(wg), sph, abortp, 20, limit);   // warp-uniform: the loads below are collective
             if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 7, i, blockIdx.x); break; }
             tc_fence_after();
             const int nvalid = (i == T - 1) ? nvalid_last : kBlock;      // >= 1; < 128 only for a ragged last block
@@ -573,7 +580,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             float r_prev = -INFINITY, r_now = mx;
             bool grow = false;
             if (i > 0) {
-                ok = mbar_wait_warp(bar_ref((i - 1) % kRefSlots, quarter), uint32_t((i - 1) / kRefSlots) & 1u, abortp, 0);
+                ok = mbar_wait_warp(bar_ref((i - 1) % kRefSlots, quarter), uint32_t((i - 1) / kRefSlots) & 1u, abortp, 0, limit);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 10, i, blockIdx.x); break; }
                 r_prev = r_pub[(i - 1) % kRefSlots][r_loc];
                 grow = mx > r_prev + kRescaleThreshold;
@@ -590,7 +597,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
                 p_free = true;
                 // O must be quiescent: P V of step i-1 (the other group's) complete.  P V is issued in step order
                 // and that of step i cannot start before this group delivers P_i.
-                ok = mbar_wait_warp(bar_pvdone(wg ^ 1), uint32_t((i - 1) >> 1) & 1u, abortp, 0);
+                ok = mbar_wait_warp(bar_pvdone(wg ^ 1), uint32_t((i - 1) >> 1) & 1u, abortp, 0, limit);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 9, i, blockIdx.x); break; }
                 tc_fence_after();
                 const float f = ex2_approx(r_prev - r_now);          // 1 for rows that did not move
@@ -622,7 +629,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
                 }
             }
             if (!p_free) {      // the one P buffer is free once P V of step i-1 (the other group's) has read it
-                ok = mbar_wait_warp(bar_pvdone(wg ^ 1), uint32_t((i - 1) >> 1) & 1u, abortp, 0);
+                ok = mbar_wait_warp(bar_pvdone(wg ^ 1), uint32_t((i - 1) >> 1) & 1u, abortp, 0, limit);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 12, i, blockIdx.x); break; }
             }
 #pragma unroll
@@ -641,11 +648,11 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
             fin[wg][0][r_loc] = m_w;
             fin[wg][1][r_loc] = l_w;
             mbar_arrive_warp(bar_fin(quarter));
-            ok = mbar_wait_warp(bar_fin(quarter), 0, abortp, 0);
+            ok = mbar_wait_warp(bar_fin(quarter), 0, abortp, 0, limit);
             if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 11, T, blockIdx.x);
         }
         if (ok) {
-            ok = mbar_wait_warp(bar_o, 0, abortp, 20);
+            ok = mbar_wait_warp(bar_o, 0, abortp, 20, limit);
             if (!ok && lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 8, T, blockIdx.x);
         }
         if (ok) {
@@ -683,6 +690,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap mapK, const __grid_const
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
+}
+
+// Self-test of the bounded wait: one warp waits on a barrier that nothing ever arms, with the limit the caller gives,
+// and must come back with CARNATOR_ERR_DEVICE_TIMEOUT in the header (same helpers as the kernels above).
+__global__ void wait_timeout_selftest_kernel(WsHeader* hdr, unsigned long long limit_ns) {
+    __shared__ __align__(8) unsigned long long bar_mem;
+    __shared__ int abort_flag;
+    const uint32_t bar = smem_u32(&bar_mem);
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        mbar_init(bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait_warp(bar, 0, &abort_flag, 50, limit_ns);
+    if (!ok && threadIdx.x == 0) set_status(hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 90, 0, 0);
 }
 
 // ---- host side ------------------------------------------------------------------------------------

@@ -949,6 +949,18 @@ extern "C" carnator_status carnator_query_status(void* ws, void* stream_) {
     return CARNATOR_OK;
 }
 
+extern "C" carnator_status carnator_selftest_wait_timeout(void* ws, uint64_t limit_ns, void* stream_) {
+    if (!ws || !aligned(ws, 256)) return CARNATOR_ERR_WORKSPACE;
+    if (limit_ns == 0 || limit_ns > kDefaultWaitNs) return CARNATOR_ERR_INVALID_ARG;
+    carnator_status st = check_device();
+    if (st != CARNATOR_OK) return st;
+    cudaStream_t stream = static_cast<cudaStream_t>(stream_);
+    CUDA_TRY(cudaMemsetAsync(ws, 0, sizeof(WsHeader), stream));
+    tc::wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(static_cast<WsHeader*>(ws), limit_ns);
+    LAUNCH_CHECK("wait_timeout_selftest_kernel");
+    return CARNATOR_OK;
+}
+
 extern "C" const char* carnator_status_string(carnator_status s) {
     switch (s) {
         case CARNATOR_OK: return "ok";

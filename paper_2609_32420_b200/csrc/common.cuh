@@ -11,6 +11,7 @@ namespace carnator {
 constexpr int kMaxKeyBlocksBuilder = 4096;   // select kernel sorts one row in shared memory
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr unsigned long long kDefaultWaitNs = 2000000000ull;   // limit of a bounded device-side wait unless the header says otherwise
 
 // First 256 bytes of every workspace.
 struct WsHeader {
@@ -18,7 +19,9 @@ struct WsHeader {
     int32_t info[3];             // where a bounded wait gave up / which check failed
     unsigned long long tiles;    // evaluated (query block, key block) pairs after compaction
     int32_t work[4];             // work-item counters of persistent kernels (zeroed with the header)
-    int32_t pad[54];
+    unsigned long long wait_limit_ns;   // 0: the default limit of every bounded device-side wait; tests set a short one
+    int32_t debug_withhold;      // 0 except in the test of the time-out path: the K producer withholds one copy
+    int32_t pad[51];
 };
 static_assert(sizeof(WsHeader) == 256, "header is 256 bytes");
 

@@ -254,6 +254,50 @@ def test_malformed_lists_are_reported_and_the_context_stays_usable(impl, fault):
     check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "after a reported list fault")
 
 
+def test_bounded_wait_runs_out_and_reports_a_timeout():
+    """The wait helper of the kernels on a barrier that nothing arms, limit 1 ms: the kernel must return by itself with
+    CARNATOR_ERR_DEVICE_TIMEOUT in the header, and the device must work afterwards."""
+    ws = torch.zeros(256, dtype=torch.uint8, device="cuda")
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    cn.selftest_wait_timeout(ws, 1_000_000)
+    t1.record()
+    assert cn.query_status(ws) == cn.ERR_DEVICE_TIMEOUT
+    assert cn.query_status(ws) == cn.OK
+    assert t0.elapsed_time(t1) < 500.0                 # gave up after about the limit, not after the 2 s default
+    assert float(torch.ones(4, device="cuda").sum()) == 4.0
+
+
+def test_withheld_tile_makes_the_attention_kernel_time_out_drain_and_return():
+    """Host-made failure inside the real kernel: the header asks the K producer of the first query block to withhold its
+    first copy and sets the limit of every wait to 2 ms.  The roles waiting on that tile must give up, the CTA must drain
+    and free its tensor memory, the call must report CARNATOR_ERR_DEVICE_TIMEOUT, and a second, clean call on the same
+    buffers must match the oracle."""
+    rng = np.random.default_rng(22)
+    B, H, N, D = 1, 1, 512, 128
+    Qb, Kb, Vb = (rand_bits(rng, (B, H, N, D)) for _ in range(3))
+    Q, K, V = to_dev(Qb), to_dev(Kb), to_dev(Vb)
+    shape = cn.make_shape(B, H, N, D, 0, 1, 1, N, 128, 128, Q, K, V, None, attn_impl=cn.IMPL_TCGEN05)
+    mask = torch.ones((B, H, 4, 4), dtype=torch.uint8, device="cuda")
+    ws = cn.compact_mask(mask, None, shape)             # clears the header: default limit, nothing withheld
+    hdr64 = ws[:256].view(torch.int64)
+    hdr32 = ws[:256].view(torch.int32)
+    hdr64[cn.HDR_WAIT_LIMIT_NS // 8] = 2_000_000
+    hdr32[cn.HDR_DEBUG_WITHHOLD // 4] = 1
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    cn.sparse_attn_compacted(Q, K, V, shape, ws)
+    t1.record()
+    assert cn.query_status(ws) == cn.ERR_DEVICE_TIMEOUT
+    assert "device status" in cn.last_cuda_error()
+    assert t0.elapsed_time(t1) < 1000.0
+    ws = cn.compact_mask(mask, None, shape, ws=ws)      # same buffers, header reset
+    O, L = cn.sparse_attn_compacted(Q, K, V, shape, ws)
+    assert cn.query_status(ws) == cn.OK
+    O_ref, L_ref = orc.attention_full(Qb, Kb, Vb, N, 128, 128, 1.0 / np.sqrt(D), mask.cpu().numpy(), None)
+    check_attention(o_to_host(O), L.cpu().numpy(), O_ref, L_ref, "after a reported time-out")
+
+
 @pytest.mark.parametrize("name,kw", [("wan1p3b_480p", {}), ("tiny", {"B": 2})], ids=["wan1p3b_two_head_chunks", "tiny_two_batch_entries"])
 def test_host_buffer_call_equals_device_call(name, kw):
     """carnator_sparse_attn_host works through the heads in chunks on its own copy streams; the result must be
