@@ -750,6 +750,20 @@ inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, in
     return r == CUDA_SUCCESS;
 }
 
+// 2-D map over a row-major [rows, D] bf16 array: box = 64 x box_rows, 128-byte swizzle, rows past the end read as zero.
+inline bool make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int D, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {cuuint64_t(D), cuuint64_t(rows)};
+    cuuint64_t strides[1] = {cuuint64_t(D) * 2};
+    cuuint32_t box[2] = {64, cuuint32_t(box_rows)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 }  // namespace tc
 
 // A tensor map cannot express a zero stride, so a tensor that is shared over heads or batch entries (stride 0 on an

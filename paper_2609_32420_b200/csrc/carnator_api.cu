@@ -134,33 +134,38 @@ carnator_status sm_count(int* out) {
 
 constexpr size_t kMaxDynamicSmem = 227 * 1024;
 
-template <int D, int NPL, int R>
-carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap& mq, const CUtensorMap& mk, int nkb, int sms, cudaStream_t stream) {
-    const size_t smem = FusedSmem<D, R>::bytes(nkb);
-    carnator_status st = allow_smem(build_fused_kernel<D, NPL, R>, smem);
+template <int D, int NPL>
+carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap (&maps)[4], int nkb, int sms, cudaStream_t stream) {
+    const size_t smem = FusedSmem<D>::bytes(nkb, fa.nkb_pad);
+    carnator_status st = allow_smem(build_fused_kernel<D, NPL>, smem);
     if (st != CARNATOR_OK) return st;
-    // the register hand-over inside the kernel (setmaxnreg) only completes if the CTA owns 256 x 32 + 512 x 104 registers
+    // the register hand-over inside the kernel (setmaxnreg) only completes if the CTA owns 256 x 40 + 512 x 96 registers
     cudaFuncAttributes attr;
-    CUDA_TRY(cudaFuncGetAttributes(&attr, build_fused_kernel<D, NPL, R>));
-    if (attr.numRegs * kFusedThreads < 256 * 32 + 512 * 104) {
+    CUDA_TRY(cudaFuncGetAttributes(&attr, build_fused_kernel<D, NPL>));
+    if (attr.numRegs * kFusedThreads < 256 * 40 + 512 * 96) {
         snprintf(g_cuda_error, sizeof(g_cuda_error), "build_fused_kernel was built with %d registers per thread: too few for its setmaxnreg split", attr.numRegs);
         return CARNATOR_ERR_UNSUPPORTED;
     }
-    build_fused_kernel<D, NPL, R><<<sms, kFusedThreads, smem, stream>>>(mq, mk, fa);
+    build_fused_kernel<D, NPL><<<sms, kFusedThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], fa);
     LAUNCH_CHECK("build_fused_kernel");
     return CARNATOR_OK;
 }
 
-// a warp of the scoring group keeps NPL scores per row, two rows, in registers
-carnator_status launch_fused_builder(const FusedArgs& fa, const CUtensorMap& mq, const CUtensorMap& mk, int D, int nkb, int sms, cudaStream_t stream) {
+// a warp of the selection group keeps the NPL keys of its row in registers
+carnator_status launch_fused_builder(const FusedArgs& fa, const CUtensorMap (&maps)[4], int D, int nkb, int sms, cudaStream_t stream) {
     if (D == 128) {
-        if (nkb <= 32 * 8) return launch_fused_r<128, 8, kFusedRows>(fa, mq, mk, nkb, sms, stream);
-        if (nkb <= 32 * 24) return launch_fused_r<128, 24, kFusedRows>(fa, mq, mk, nkb, sms, stream);
-        return launch_fused_r<128, 32, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+        if (nkb <= 32 * 8) return launch_fused_r<128, 8>(fa, maps, nkb, sms, stream);
+        if (nkb <= 32 * 20) return launch_fused_r<128, 20>(fa, maps, nkb, sms, stream);
+        return launch_fused_r<128, 32>(fa, maps, nkb, sms, stream);
     }
-    if (nkb <= 32 * 8) return launch_fused_r<64, 8, kFusedRows>(fa, mq, mk, nkb, sms, stream);
-    if (nkb <= 32 * 24) return launch_fused_r<64, 24, kFusedRows>(fa, mq, mk, nkb, sms, stream);
-    return launch_fused_r<64, 32, kFusedRows>(fa, mq, mk, nkb, sms, stream);
+    if (nkb <= 32 * 8) return launch_fused_r<64, 8>(fa, maps, nkb, sms, stream);
+    if (nkb <= 32 * 20) return launch_fused_r<64, 20>(fa, maps, nkb, sms, stream);
+    return launch_fused_r<64, 32>(fa, maps, nkb, sms, stream);
+}
+
+size_t fused_smem_bytes(int D, int nkb) {
+    const int pad = (nkb + 3) & ~3;
+    return D == 128 ? FusedSmem<128>::bytes(nkb, pad) : FusedSmem<64>::bytes(nkb, pad);
 }
 }  // namespace
 
@@ -222,7 +227,8 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
     int sms = 0;
     st = sm_count(&sms);
     if (st != CARNATOR_OK) return st;
-    const bool fused_able = p->mode == CARNATOR_MODE_TOPK && nkb <= 32 * 32 && tma_strides_ok(s, s->q_stride) && tma_strides_ok(s, s->k_stride);
+    const bool fused_able = p->mode == CARNATOR_MODE_TOPK && nkb <= 32 * 32 && tma_strides_ok(s, s->q_stride) && tma_strides_ok(s, s->k_stride) &&
+                            fused_smem_bytes(s->D, nkb) <= kMaxDynamicSmem;
     const bool fused_pays = int64_t(s->B) * s->H * ceil_div(nqb, kFusedRows) >= 2 * int64_t(sms);
     const int choice = g_builder_path.load();
     if (fused_able && (choice == 2 || (choice == 0 && fused_pays))) {
@@ -230,14 +236,20 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
         FusedArgs fa;
         fa.pool = pa; fa.sel = sa;
         fa.scores_out = pooled_scores_opt; fa.done = w.done; fa.hdr = w.hdr;
+        fa.split[0] = w.qsplit; fa.split[1] = w.ksplit;
         fa.B = s->B; fa.scale = effective_scale(s);
-        CUtensorMap mq, mk;      // one box = 64 elements x one block of tokens; rows >= N read as zero
-        if (!tc::make_map(&mq, Q, s->B, s->H, s->N, s->D, s->q_stride, s->block_q) ||
-            !tc::make_map(&mk, K, s->B, s->H, s->N, s->D, s->k_stride, s->block_k)) {
+        fa.nkb_pad = (nkb + 3) & ~3;
+        CUtensorMap maps[4];     // Q, K: one box = 64 elements x one block of tokens (rows >= N read as zero); the three-term
+                                 // means of Q: 16 rows per box; of K: 128 rows per box
+        const int64_t bh = int64_t(s->B) * s->H;
+        if (!tc::make_map(&maps[0], Q, s->B, s->H, s->N, s->D, s->q_stride, s->block_q) ||
+            !tc::make_map(&maps[1], K, s->B, s->H, s->N, s->D, s->k_stride, s->block_k) ||
+            !tc::make_map_2d(&maps[2], w.qsplit, 3 * bh * nqb, s->D, kFusedRows) ||
+            !tc::make_map_2d(&maps[3], w.ksplit, 3 * bh * nkb, s->D, 128)) {
             snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed or is unavailable");
             return CARNATOR_ERR_CUDA;
         }
-        return launch_fused_builder(fa, mq, mk, s->D, nkb, sms, stream);
+        return launch_fused_builder(fa, maps, s->D, nkb, sms, stream);
     }
     // M1
     {

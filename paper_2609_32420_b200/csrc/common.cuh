@@ -50,13 +50,15 @@ inline AttnWs attn_ws_layout(void* base, int B, int H, int nqb, int nkb) {
     return w;
 }
 
-// Layout of the builder workspace: header | pooled-blocks counters | qbar | kbar | scores.
+// Layout of the builder workspace: header | pooled-blocks counters | qbar | kbar | scores | three-term means of Q, of K.
 struct BuildWs {
     WsHeader* hdr;
     int32_t* done;   // [B,H]  pooled blocks of each head written so far (fused builder; zeroed together with the header)
     float* qbar;     // [B,H,nqb,D]
     float* kbar;     // [B,H,nkb,D]
     float* scores;   // [B,H,nqb,nkb]
+    __nv_bfloat16* qsplit;   // [3][B*H*nqb][D]  block means of Q as three bf16 terms (fused builder)
+    __nv_bfloat16* ksplit;   // [3][B*H*nkb][D]
     size_t bytes;
 };
 
@@ -69,6 +71,8 @@ inline BuildWs build_ws_layout(void* base, int B, int H, int nqb, int nkb, int D
     w.qbar = reinterpret_cast<float*>(p + off);             off += align256(size_t(B) * H * nqb * D * 4);
     w.kbar = reinterpret_cast<float*>(p + off);             off += align256(size_t(B) * H * nkb * D * 4);
     w.scores = reinterpret_cast<float*>(p + off);           off += align256(size_t(B) * H * nqb * size_t(nkb) * 4);
+    w.qsplit = reinterpret_cast<__nv_bfloat16*>(p + off);   off += align256(size_t(3) * B * H * nqb * D * 2);
+    w.ksplit = reinterpret_cast<__nv_bfloat16*>(p + off);   off += align256(size_t(3) * B * H * nkb * D * 2);
     w.bytes = off;
     return w;
 }

@@ -41,7 +41,7 @@ def test_workspace_sizes():
     al = lambda x: (x + 255) // 256 * 256
     assert cn.attn_workspace_bytes(s) == 256 + 2 * al(rows * 4) + al(rows * nkb * 4)
     p = cn.BuildParams(0, 0.25, 0.9, -1, 0, 1)
-    assert cn.build_workspace_bytes(s, p) == 256 + al(1 * 2 * 4) + 2 * al(rows * 128 * 4) + al(rows * nkb * 4)
+    assert cn.build_workspace_bytes(s, p) == 256 + al(1 * 2 * 4) + 2 * al(rows * 128 * 4) + al(rows * nkb * 4) + 2 * al(3 * rows * 128 * 2)
     assert cn.attn_host_arena_bytes(s) > 4 * 2 * 1000 * 128 * 2
 
 

@@ -119,9 +119,10 @@ def test_keep_ratio_one_is_all_ones(builder_path):
 @pytest.mark.parametrize("name,kw", [("tiny", {}), ("wan1p3b_480p", dict(H=3, T=5)), ("cogvideox5b", dict(H=5, T=3)),
                                      ("hunyuan_720p", dict(H=2, T=2)), ("wan14b_720p", dict(H=3)), ("hunyuan_720p", dict(H=2))])
 def test_fused_kernel_and_three_kernel_path_agree(name, kw):
-    """Top-k mode normally runs as one persistent kernel that pools on the tensor cores; the three separate kernels pool
-    with CUDA-core sums.  The pooled scores may differ in the last bits (order of the fp32 sums), far inside the 2e-5
-    the oracle comparison allows; masks may differ only where a score sits that close to the row's threshold."""
+    """Large top-k layers run as one persistent kernel that pools and scores on the tensor cores (block means as three
+    bf16 terms, six products per score, fp32 accumulate); the three separate kernels use CUDA-core fp32 sums and FFMA
+    chains.  Both carry rounding errors of a few 1e-6 on scores of magnitude 3 to 4 (each is checked against the fp64
+    oracle to 2e-5 elsewhere); masks may differ only where a score sits that close to the row's threshold."""
     w = wl.shrunk(wl.get(name), **kw) if kw else wl.get(name)
     nthreads = min(16, os.cpu_count() or 1)
     Q = to_dev(wl.gen_tensor(w, "Q", "history", threads=nthreads))
@@ -141,7 +142,7 @@ def test_fused_kernel_and_three_kernel_path_agree(name, kw):
     finally:
         cn.debug_set_builder_path(cn.BUILDER_AUTO)
     (m0, s0), (m1, s1) = out
-    assert float((s0 - s1).abs().max()) <= 5e-6
+    assert float((s0 - s1).abs().max()) <= 1e-5
     assert bool((m0.sum(-1) == m1.sum(-1)).all())                       # top-k: same number of blocks per row
     assert int((m0 != m1).sum()) <= 1e-5 * m0.numel() + 2
 
