@@ -269,6 +269,14 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
          | (1ull << 46)
          | (2ull << 61);
 }
+// Same with the 64-byte swizzle (rows of 64 B, atoms of 8 rows = 512 B): layout type 4.
+__device__ __forceinline__ uint64_t smem_desc_sw64(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+    return uint64_t((addr & 0x3FFFFu) >> 4)
+         | (uint64_t((lbo_bytes >> 4) & 0x3FFFu) << 16)
+         | (uint64_t((sbo_bytes >> 4) & 0x3FFFu) << 32)
+         | (1ull << 46)
+         | (4ull << 61);
+}
 // Instruction descriptor for kind::f16: fp32 accumulator, bf16 x bf16, M x N, B operand major-ness.
 __host__ __device__ constexpr uint32_t instr_desc(int M, int N, int b_mn_major) {
     return (1u << 4) | (1u << 7) | (1u << 10) | (uint32_t(b_mn_major) << 16) | (uint32_t(N >> 3) << 17) | (uint32_t(M >> 4) << 24);
@@ -750,17 +758,18 @@ inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, in
     return r == CUDA_SUCCESS;
 }
 
-// 2-D map over a row-major [rows, D] bf16 array: box = 64 x box_rows, 128-byte swizzle, rows past the end read as zero.
-inline bool make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int D, int box_rows) {
+// 2-D map over a row-major [rows, D] bf16 array: box = box_cols x box_rows (64 columns: 128-byte swizzle, 32 columns:
+// 64-byte swizzle), rows past the end read as zero.
+inline bool make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int D, int box_rows, int box_cols = 64) {
     EncodeTiledFn fn = encode_fn();
     if (!fn) return false;
     cuuint64_t dims[2] = {cuuint64_t(D), cuuint64_t(rows)};
     cuuint64_t strides[1] = {cuuint64_t(D) * 2};
-    cuuint32_t box[2] = {64, cuuint32_t(box_rows)};
+    cuuint32_t box[2] = {cuuint32_t(box_cols), cuuint32_t(box_rows)};
     cuuint32_t estr[2] = {1, 1};
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, box_cols == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 

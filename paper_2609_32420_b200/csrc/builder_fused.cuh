@@ -36,8 +36,9 @@ constexpr int kFusedThreads = kFusedPoolThreads + kFusedScoreThreads;
 constexpr int kFusedStages = 3;       // blocks in the pooling ring
 constexpr int kFusedBatch = 4;        // pooling items taken per counter update; L2 is asked for one batch ahead
 constexpr int kFusedQueue = 8;        // decoded items in flight between producer and epilogue (> kFusedStages + 2)
-constexpr int kFusedRows = 16;        // query blocks per scoring item (N of the score products; one per selection warp)
-constexpr int kFusedTmemCols = 512;   // [0, 32): two pooling accumulators; [128, 512): score tiles, 16 columns per accumulator
+constexpr int kFusedRows = 16;        // query blocks per scoring item (N of the score products; one selection warp each)
+constexpr int kFusedAStages = 2;      // buffers of the key-block operand of the score products
+constexpr int kFusedTmemCols = 512;   // [0, 32): two pooling accumulators; [32, 512): score tiles
 
 struct FusedArgs {
     PoolArgs pool;
@@ -91,20 +92,22 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 }
 
 // Shared-memory plan.  Pooling ring: blocks of 128 token rows as D/64 boxes (128 rows x 128 B, 128-byte swizzle).
-// Score operands: A = the three terms of 128 key-block means, one 64-element half of the head dimension at a time
-// (3 boxes of 128 rows x 128 B); B = the three terms of the item's 16 query-block means, both halves (6 boxes of
-// 16 rows x 128 B).
+// Score operands: A = the three terms of 128 key-block means, one 32-element quarter of the head dimension at a time
+// (3 boxes of 128 rows x 64 B, 64-byte swizzle), two buffers; B = the three terms of the item's 16 query-block means,
+// whole rows (boxes of 16 rows x 128 B, 128-byte swizzle).
 template <int D>
 struct FusedSmem {
     static constexpr size_t kBox = size_t(128) * 128;
+    static constexpr size_t kBoxB = size_t(kFusedRows) * 128;                     // 16 query blocks x 64 elements
     static constexpr size_t kSlot = (D / 64) * kBox;
     static constexpr size_t kOffRing = 0;                                         // 1 KiB aligned
-    static constexpr size_t kOffScoreA = kOffRing + kFusedStages * kSlot;         // 3 x 16 KiB
-    static constexpr size_t kOffScoreB = kOffScoreA + 3 * kBox;                   // 3 terms x D/64 halves x 2 KiB
-    static constexpr size_t kOffOnes = kOffScoreB + 3 * (D / 64) * 2048;          // 16 rows x 128 B of bf16 ones
+    static constexpr size_t kBoxA = size_t(128) * 64;                             // 128 key blocks x 32 elements, 64-byte swizzle
+    static constexpr size_t kOffScoreA = kOffRing + kFusedStages * kSlot;         // kFusedAStages buffers x 3 terms x 8 KiB
+    static constexpr size_t kOffScoreB = kOffScoreA + kFusedAStages * 3 * kBoxA;  // 3 terms x D/64 halves x 2 KiB
+    static constexpr size_t kOffOnes = kOffScoreB + 3 * (D / 64) * kBoxB;         // 16 rows x 128 B of bf16 ones
     static constexpr size_t kOffBar = kOffOnes + 2048;                            // mbarriers
-    static constexpr size_t kOffFrames = kOffBar + 256;                           // int2 [nkb]
-    __host__ __device__ static size_t off_scores(int nkb) { return (kOffFrames + size_t(nkb) * 8 + 15) & ~size_t(15); }
+    static constexpr size_t kOffScores = kOffBar + 256;                           // float [RP][nkb_pad]
+    __host__ __device__ static size_t off_scores(int) { return kOffScores; }
     static size_t bytes(int nkb, int nkb_pad) { return off_scores(nkb) + size_t(kFusedRows) * nkb_pad * 4 + 1024; }   // + slack to align the base
 };
 
@@ -117,8 +120,11 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     __shared__ ScoreItem score_q[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
+    constexpr int NR = kFusedRows, RP = kFusedRows;                 // query blocks per item = rows selected at once
     using L = FusedSmem<D>;
     constexpr int KH = D / 64;                                         // 64-element halves of the head dimension
+    // accumulators per score tile: the large product t1 t1, one per half of the head dimension, apart from the five small ones
+    constexpr int NACC = KH + 1;
     const int tid = threadIdx.x, warp_id = tid >> 5, lane = tid & 31;
     const int nqb = a.sel.nqb, nkb = a.sel.nkb, H = a.sel.H;
     const int heads = a.B * H;
@@ -131,7 +137,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     auto bar_acc = [&](int s) { return bars + 64 + 8 * s; };         // pooling accumulator s holds fresh sums
     auto bar_accfree = [&](int s) { return bars + 80 + 8 * s; };     // the epilogue has read accumulator s
     const uint32_t bar_drain = bars + 96, bar_drain2 = bars + 104;
-    const uint32_t bar_afull = bars + 112, bar_afree = bars + 120;   // score operand A (key-block means, one half)
+    auto bar_afull = [&](int s) { return bars + 160 + 8 * s; };      // score operand A, buffer s (key-block means, one quarter)
+    auto bar_afree = [&](int s) { return bars + 192 + 8 * s; };
     const uint32_t bar_bfull = bars + 128, bar_bfree = bars + 136;   // score operand B (the item's query-block means)
     const uint32_t bar_sfull = bars + 144, bar_sfree = bars + 152;   // the item's scores in tensor memory
     volatile int* abortp = &abort_flag;
@@ -141,7 +148,7 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         for (int s = 0; s < kFusedStages; ++s) { tc::mbar_init(bar_full(s), 1); tc::mbar_init(bar_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { tc::mbar_init(bar_acc(s), 1); tc::mbar_init(bar_accfree(s), 4); }
         tc::mbar_init(bar_drain, 1); tc::mbar_init(bar_drain2, 1);
-        tc::mbar_init(bar_afull, 1); tc::mbar_init(bar_afree, 1);
+        for (int s = 0; s < kFusedAStages; ++s) { tc::mbar_init(bar_afull(s), 1); tc::mbar_init(bar_afree(s), 1); }
         tc::mbar_init(bar_bfull, 1); tc::mbar_init(bar_bfree, 1);
         tc::mbar_init(bar_sfull, 1); tc::mbar_init(bar_sfree, kFusedScoreThreads / 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -156,10 +163,10 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem = tmem_slot;
-    const uint32_t tmem_s = tmem + 128;                               // score tiles
+    const uint32_t tmem_s = tmem + 32;                                // score tiles (behind the two pooling accumulators)
     const int per_head = nqb + nkb;
     const int pool_total = heads * per_head;
-    const int groups_per_head = (nqb + kFusedRows - 1) / kFusedRows;
+    const int groups_per_head = (nqb + NR - 1) / NR;
     const int score_total = heads * groups_per_head;
 
     // Register budget: 768 threads x 80 at launch; the pooling and operand warps keep 40 each, the selection group takes
@@ -313,7 +320,7 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 }
                 if (item >= score_total) { score_q[n & 3] = si; tc::mbar_arrive(bar_bfull); break; }
                 si.bh = item / groups_per_head;
-                si.I0 = (item - si.bh * groups_per_head) * kFusedRows;
+                si.I0 = (item - si.bh * groups_per_head) * NR;
                 if (si.bh != ready_head) {                              // the head's pooled vectors must all be written
                     if (ld_acquire(a.done + si.bh) < per_head) {
                         const unsigned long long t0 = global_timer_ns();
@@ -330,33 +337,36 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     asm volatile("fence.proxy.async.global;" ::: "memory");
                 }
                 score_q[n & 3] = si;
-                tc::mbar_expect_tx(bar_bfull, uint32_t(3 * KH * 2048));
+                tc::mbar_expect_tx(bar_bfull, uint32_t(3 * KH * L::kBoxB));
                 for (int t3 = 0; t3 < 3; ++t3)
                     for (int kh = 0; kh < KH; ++kh)
-                        tma_load_2d(smem_base + uint32_t(L::kOffScoreB + (t3 * KH + kh) * 2048), &mapQs, bar_bfull,
+                        tma_load_2d(smem_base + uint32_t(L::kOffScoreB + (t3 * KH + kh) * L::kBoxB), &mapQs, bar_bfull,
                                     kh * 64, t3 * rows_q + si.bh * nqb + si.I0);
                 for (int t = 0; t < ntiles && ok; ++t)
-                    for (int kh = 0; kh < KH; ++kh, ++step) {
-                        if (step >= 1) {
-                            ok = tc::mbar_wait(bar_afree, uint32_t(step - 1) & 1u, abortp, 32);
+                    for (int kq = 0; kq < 2 * KH; ++kq, ++step) {        // quarters of 32 elements, the buffers in turn
+                        const int buf = step % kFusedAStages;
+                        if (step >= kFusedAStages) {
+                            ok = tc::mbar_wait(bar_afree(buf), uint32_t(step / kFusedAStages - 1) & 1u, abortp, 32);
                             if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 46, step, blockIdx.x); *abortp = 1; break; }
                         }
-                        tc::mbar_expect_tx(bar_afull, uint32_t(3 * L::kBox));
+                        tc::mbar_expect_tx(bar_afull(buf), uint32_t(3 * L::kBoxA));
                         for (int t3 = 0; t3 < 3; ++t3)
-                            tma_load_2d(smem_base + uint32_t(L::kOffScoreA + t3 * L::kBox), &mapKs, bar_afull,
-                                        kh * 64, t3 * rows_k + si.bh * nkb + t * 128);
+                            tma_load_2d(smem_base + uint32_t(L::kOffScoreA + (buf * 3 + t3) * L::kBoxA), &mapKs, bar_afull(buf),
+                                        kq * 32, t3 * rows_k + si.bh * nkb + t * 128);
                     }
             }
             // on the way out after an abort, copies in flight must land first; an unarmed barrier simply runs out
-            if (*abortp) { tc::mbar_wait_drain(bar_afull, uint32_t(step > 0 ? step - 1 : 0) & 1u, 20000000ull); }
+            if (*abortp)
+                for (int k = 1; k <= kFusedAStages && step - k >= 0; ++k)
+                    tc::mbar_wait_drain(bar_afull((step - k) % kFusedAStages), uint32_t((step - k) / kFusedAStages) & 1u, 20000000ull);
         }
     } else if (warp_id == 7) {
         // ================= scores on the tensor cores =================
         if (lane == 0) {
             // S^T tile t (128 key blocks x 16 query blocks) += A_term x B_term^T over the six term pairs, 16 elements of
             // the head dimension per instruction; both operands K-major (rows of 128 B, 128-byte swizzle).
-            constexpr uint32_t idesc = tc::instr_desc(128, kFusedRows, 0);
-            const uint64_t da0 = tc::smem_desc(smem_base + uint32_t(L::kOffScoreA), 16, 1024);
+            constexpr uint32_t idesc = tc::instr_desc(128, NR, 0);
+            const uint64_t da0 = tc::smem_desc_sw64(smem_base + uint32_t(L::kOffScoreA), 16, 512);
             const uint64_t db0 = tc::smem_desc(smem_base + uint32_t(L::kOffScoreB), 16, 1024);
             constexpr int pa[6] = {0, 0, 1, 0, 1, 2}, pb[6] = {0, 1, 0, 2, 1, 0};       // term pairs, largest products first
             int step = 0;
@@ -371,24 +381,27 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 }
                 if (si.bh < 0) { tc::mbar_arrive(bar_sfull); break; }                   // pass the end marker on
                 for (int t = 0; t < ntiles && ok; ++t)
-                    for (int kh = 0; kh < KH; ++kh, ++step) {
-                        ok = tc::mbar_wait(bar_afull, uint32_t(step) & 1u, abortp, 32);
+                    for (int kq = 0; kq < 2 * KH; ++kq, ++step) {
+                        const int buf = step % kFusedAStages, kh = kq >> 1;
+                        ok = tc::mbar_wait(bar_afull(buf), uint32_t(step / kFusedAStages) & 1u, abortp, 32);
                         if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 49, step, blockIdx.x); *abortp = 1; break; }
                         tc::tc_fence_after();
                         // The tensor cores add into an fp32 accumulator without guard bits, so a long chain of additions
                         // at the magnitude of the score loses a few bits.  The leading product t1 t1 (the only large one)
-                        // therefore gets an accumulator per half of the head dimension (four additions each); the five
-                        // small products share a third one.  The selection group adds the three in fp32.
-                        const uint32_t d_tile = tmem_s + uint32_t(t * kFusedRows * (KH + 1));
+                        // therefore has an accumulator per half of the head dimension (four additions each); the five
+                        // small products share another.  The selection group adds them in fp32.
+                        const uint32_t d_tile = tmem_s + uint32_t(t * NR * NACC);
+                        const uint32_t d_big = d_tile + uint32_t((NACC == 2 ? 0 : kh) * NR), d_small = d_tile + uint32_t((NACC - 1) * NR);
+                        const bool big_first = NACC == 2 ? kq == 0 : (kq & 1) == 0;
 #pragma unroll
                         for (int p = 0; p < 6; ++p)
 #pragma unroll
-                            for (int kk = 0; kk < 4; ++kk)
-                                tc::mma_ss(p == 0 ? d_tile + uint32_t(kh * kFusedRows) : d_tile + uint32_t(KH * kFusedRows),
-                                           da0 + uint64_t((pa[p] * L::kBox + kk * 32) >> 4),
-                                           db0 + uint64_t(((pb[p] * KH + kh) * 2048 + kk * 32) >> 4),
-                                           idesc, p == 0 ? (kk > 0 ? 1u : 0u) : ((kh > 0 || p > 1 || kk > 0) ? 1u : 0u));
-                        tc::tc_commit(bar_afree);
+                            for (int kk = 0; kk < 2; ++kk)
+                                tc::mma_ss(p == 0 ? d_big : d_small,
+                                           da0 + uint64_t(((buf * 3 + pa[p]) * L::kBoxA + kk * 32) >> 4),
+                                           db0 + uint64_t(((pb[p] * KH + kh) * L::kBoxB + (kq & 1) * 64 + kk * 32) >> 4),
+                                           idesc, p == 0 ? ((!big_first || kk > 0) ? 1u : 0u) : ((kq > 0 || p > 1 || kk > 0) ? 1u : 0u));
+                        tc::tc_commit(bar_afree(buf));
                     }
                 if (!ok) break;
                 tc::tc_commit(bar_bfree);
@@ -404,13 +417,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     constexpr int NT = kFusedScoreThreads;
     constexpr int NW = NT / 32;                                        // 16 warps = kFusedRows: one query block per warp
     static_assert(NW == kFusedRows, "one selection warp per row of an item");
-    int2* kframes = reinterpret_cast<int2*>(fsm + L::kOffFrames);
-    float* sS = reinterpret_cast<float*>(fsm + L::off_scores(nkb));  // [kFusedRows][nkb_pad]
+    float* sS = reinterpret_cast<float*>(fsm + L::off_scores(nkb));  // [RP][nkb_pad]
     const Geometry g = a.sel.g;
-    for (int J = t; J < nkb; J += NT) {
-        const int k_lo = max(J * g.bk, g.n_text), k_hi = min(g.N, (J + 1) * g.bk) - 1;
-        kframes[J] = (k_hi >= k_lo) ? make_int2((k_lo - g.n_text) / g.hw, (k_hi - g.n_text) / g.hw) : make_int2(1, 0);
-    }
     const int warp = t >> 5;
     const int quarter = warp & 3;                                      // tensor-memory lanes this warp may read
     const uint32_t lane_base = uint32_t(quarter * 32) << 16;
@@ -422,48 +430,71 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         const ScoreItem si = score_q[n & 3];
         if (si.bh < 0) break;
         const int bh = si.bh, I0 = si.I0;
-        const int nrows = min(kFusedRows, nqb - I0);
-        // ---- tensor memory -> shared memory rows: a thread holds one key block's scores against the item's 16 query blocks ----
+        const int nrows = min(NR, nqb - I0);
         tc::tc_fence_after();
-        for (int tile = warp >> 2; tile < ntiles; tile += NW / 4) {
-            float v[16], u[16];
-            tmem_ld16(tmem_s + lane_base + uint32_t(tile * kFusedRows * (KH + 1)), v);                  // t1 t1, first half of d
-            tmem_ld16(tmem_s + lane_base + uint32_t(tile * kFusedRows * (KH + 1) + KH * kFusedRows), u);   // the small products
-            tc::tmem_wait_ld();
-            if (KH == 2) {
-                float v2[16];
-                tmem_ld16(tmem_s + lane_base + uint32_t(tile * kFusedRows * (KH + 1) + kFusedRows), v2);  // t1 t1, second half
-                tc::tmem_wait_ld();
+        constexpr int TPW = 2;                                         // score tiles a warp reads at most (8 tiles, 4 warps per lane quarter)
+        float v[TPW][16];                                              // with 8-row passes an even pass reads for the odd one after it as well
+        constexpr int kLastRead = RP == 16 ? NR / RP - 1 : NR / RP - 2;
+#pragma unroll 1
+        for (int pass = 0; pass < NR / RP; ++pass) {
+        // ---- tensor memory -> registers: a thread holds one key block's scores against 16 of the item's query blocks ----
+        const int c0 = ((pass * RP) / 16) * 16;                        // first of the 16 accumulator columns read in this pass
+        if (RP == 16 || (pass & 1) == 0) {
 #pragma unroll
-                for (int i = 0; i < 16; ++i) v[i] += v2[i];
-            }
+            for (int j = 0; j < TPW; ++j) {
+                const int tile = (warp >> 2) + j * (NW / 4);
+                if (tile < ntiles) {                                   // warp-uniform
+                    float u[16];
+                    tmem_ld16(tmem_s + lane_base + uint32_t(tile * NR * NACC + c0), v[j]);                        // t1 t1 (first half of d)
+                    tmem_ld16(tmem_s + lane_base + uint32_t(tile * NR * NACC + (NACC - 1) * NR + c0), u);         // the small products
+                    tc::tmem_wait_ld();
+                    if (NACC == 3) {
+                        float v2[16];
+                        tmem_ld16(tmem_s + lane_base + uint32_t(tile * NR * NACC + NR + c0), v2);                  // t1 t1, second half
+                        tc::tmem_wait_ld();
 #pragma unroll
-            for (int i = 0; i < 16; ++i) v[i] += u[i];
-            const int J = tile * 128 + quarter * 32 + lane;
-            if (J < nkb) {
+                        for (int i = 0; i < 16; ++i) v[j][i] += v2[i];
+                    }
 #pragma unroll
-                for (int i = 0; i < kFusedRows; ++i) sS[i * a.nkb_pad + J] = a.scale * v[i];
+                    for (int i = 0; i < 16; ++i) v[j][i] = a.scale * (v[j][i] + u[i]);
+                }
             }
         }
-        tc::tc_fence_before();
-        tc::mbar_arrive_warp(bar_sfree);                               // the next item's products may overwrite the tiles
+        if (pass == kLastRead) {       // the last columns are in registers: the next item's products may overwrite the tiles
+            tc::tc_fence_before();
+            tc::mbar_arrive_warp(bar_sfree);
+        }
+        // ---- RP rows into shared memory (one row per query block), then one warp per row selects ----
+#pragma unroll
+        for (int j = 0; j < TPW; ++j) {
+            const int tile = (warp >> 2) + j * (NW / 4);
+            const int J = tile * 128 + quarter * 32 + lane;
+            if (tile < ntiles && J < nkb) {
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (RP == 16 || i / 8 == (pass & 1)) sS[(i % RP) * a.nkb_pad + J] = v[j][i];
+            }
+        }
         named_bar(2, NT);
-        // ---- selection: one warp per query block ----
-        if (warp < nrows) {
-            const int I = I0 + warp;
+        const int rsel = pass * RP + warp;                              // row of the item this warp selects for
+        if (warp < RP && rsel < nrows) {
+            const int I = I0 + rsel;
             const float* srow = sS + warp * a.nkb_pad;
             const int64_t row = (int64_t(bh) * nqb + I) * nkb;
             const bool text_row = g.text_dense && g.n_text > 0 && I * g.bq < g.n_text;
-            int f_lo = 0, f_hi = 0;
-            bool has_window = false;
+            // Always-kept key blocks of the frame window: blocks are runs of consecutive tokens, so the blocks that touch
+            // frames [f_lo, f_hi] are the interval [j_lo, j_hi] of blocks that touch tokens [n_text + f_lo hw, n_text + (f_hi + 1) hw).
+            int j_lo = 1, j_hi = 0;
             if (g.window >= 0) {
                 const int q_lo = max(I * g.bq, g.n_text), q_hi = min(g.N, (I + 1) * g.bq) - 1;
                 if (q_hi >= q_lo) {
-                    has_window = true;
-                    f_lo = max(0, (q_lo - g.n_text) / g.hw - g.window);
-                    f_hi = min(g.T - 1, (q_hi - g.n_text) / g.hw + g.window);
+                    const int f_lo = max(0, (q_lo - g.n_text) / g.hw - g.window);
+                    const int f_hi = min(g.T - 1, (q_hi - g.n_text) / g.hw + g.window);
+                    j_lo = (g.n_text + f_lo * g.hw) / g.bk;
+                    j_hi = (min(g.N, g.n_text + (f_hi + 1) * g.hw) - 1) / g.bk;
                 }
             }
+            if (text_row) { j_lo = 0; j_hi = nkb - 1; }
             uint32_t key[NPL];
             uint32_t forced_bits[(NPL + 31) / 32];
 #pragma unroll
@@ -474,12 +505,11 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 const int J = q * 32 + lane;
                 uint32_t k = 0u;                                        // always-kept and out-of-range entries never compete
                 if (J < nkb) {
-                    const float v = srow[J];
-                    const int2 kf = kframes[J];
-                    const bool forced = text_row || J < text_cols || (has_window && kf.x <= kf.y && kf.x <= f_hi && kf.y >= f_lo);
+                    const float sv = srow[J];
+                    const bool forced = J < text_cols || (J >= j_lo && J <= j_hi);
                     if (forced) { forced_bits[q >> 5] |= 1u << (q & 31); ++my_forced; }
-                    else k = ordered_bits(v);
-                    if (a.scores_out) a.scores_out[row + J] = v;
+                    else k = ordered_bits(sv);
+                    if (a.scores_out) a.scores_out[row + J] = sv;
                 }
                 key[q] = k;
             }
@@ -489,10 +519,18 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             n_admit = min(n_admit, nfree);
             // k-th largest key, bit by bit: the largest T with #(key >= T) >= n_admit.  Once a candidate is met by exactly
             // n_admit keys the kept set is known (the remaining bits would only find its smallest key).
-            uint32_t T = 0u;
+            // Bits above the first one in which two competing keys differ are the same in T as in every such key: they
+            // are taken over at once (keys of always-kept and absent blocks are 0 and never compete).
+            uint32_t k_or = 0u, k_and = 0xFFFFFFFFu;
+#pragma unroll
+            for (int q = 0; q < NPL; ++q) { k_or |= key[q]; k_and &= key[q] ? key[q] : 0xFFFFFFFFu; }
+            k_or = __reduce_or_sync(0xffffffffu, k_or);
+            k_and = __reduce_and_sync(0xffffffffu, k_and);
+            const int top = 31 - __clz(int((k_or ^ k_and) | 1u));       // highest bit in which competing keys differ (0 if none do)
+            uint32_t T = (top >= 31) ? 0u : (k_and & ~((2u << top) - 1u));
             bool exact = n_admit == 0;
 #pragma unroll 1
-            for (int bit = 31; bit >= 0 && !exact; --bit) {
+            for (int bit = top; bit >= 0 && !exact; --bit) {
                 const uint32_t cand = T | (1u << bit);
                 int c0 = 0, c1 = 0, c2 = 0, c3 = 0;
 #pragma unroll
@@ -521,7 +559,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 if (J < nkb) a.sel.mask[row + J] = keep ? 1 : 0;
             }
         }
-        named_bar(2, NT);                                              // the rows are free for the next item
+        named_bar(2, NT);                                              // the rows are free for the next pass / item
+        }
     }
     }
 

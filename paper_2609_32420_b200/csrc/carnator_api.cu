@@ -132,7 +132,7 @@ carnator_status sm_count(int* out) {
     return CARNATOR_OK;
 }
 
-constexpr size_t kMaxDynamicSmem = 227 * 1024;
+constexpr size_t kMaxDynamicSmem = 226 * 1024;     // 227 KiB per CTA less the kernels' static shared memory
 
 template <int D, int NPL>
 carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap (&maps)[4], int nkb, int sms, cudaStream_t stream) {
@@ -151,21 +151,21 @@ carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap (&maps)[4]
     return CARNATOR_OK;
 }
 
-// a warp of the selection group keeps the NPL keys of its row in registers
-carnator_status launch_fused_builder(const FusedArgs& fa, const CUtensorMap (&maps)[4], int D, int nkb, int sms, cudaStream_t stream) {
-    if (D == 128) {
-        if (nkb <= 32 * 8) return launch_fused_r<128, 8>(fa, maps, nkb, sms, stream);
-        if (nkb <= 32 * 20) return launch_fused_r<128, 20>(fa, maps, nkb, sms, stream);
-        return launch_fused_r<128, 32>(fa, maps, nkb, sms, stream);
-    }
-    if (nkb <= 32 * 8) return launch_fused_r<64, 8>(fa, maps, nkb, sms, stream);
-    if (nkb <= 32 * 20) return launch_fused_r<64, 20>(fa, maps, nkb, sms, stream);
-    return launch_fused_r<64, 32>(fa, maps, nkb, sms, stream);
+bool fused_fits(int D, int nkb) {
+    const int pad = (nkb + 3) & ~3;
+    return (D == 128 ? FusedSmem<128>::bytes(nkb, pad) : FusedSmem<64>::bytes(nkb, pad)) <= kMaxDynamicSmem;
 }
 
-size_t fused_smem_bytes(int D, int nkb) {
-    const int pad = (nkb + 3) & ~3;
-    return D == 128 ? FusedSmem<128>::bytes(nkb, pad) : FusedSmem<64>::bytes(nkb, pad);
+// a warp of the selection group keeps the NPL keys of its row in registers
+template <int D>
+carnator_status launch_fused_d(const FusedArgs& fa, const CUtensorMap (&maps)[4], int nkb, int sms, cudaStream_t stream) {
+    if (nkb <= 32 * 8) return launch_fused_r<D, 8>(fa, maps, nkb, sms, stream);
+    if (nkb <= 32 * 20) return launch_fused_r<D, 20>(fa, maps, nkb, sms, stream);
+    return launch_fused_r<D, 32>(fa, maps, nkb, sms, stream);
+}
+
+carnator_status launch_fused_builder(const FusedArgs& fa, const CUtensorMap (&maps)[4], int D, int nkb, int sms, cudaStream_t stream) {
+    return D == 128 ? launch_fused_d<128>(fa, maps, nkb, sms, stream) : launch_fused_d<64>(fa, maps, nkb, sms, stream);
 }
 }  // namespace
 
@@ -222,15 +222,15 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
     sa.g.N = s->N; sa.g.n_text = s->n_text; sa.g.hw = s->Hg * s->Wg > 0 ? s->Hg * s->Wg : 1; sa.g.T = s->T;
     sa.g.bq = s->block_q; sa.g.bk = s->block_k; sa.g.window = p->window_frames; sa.g.text_dense = p->text_dense;
 
-    // The persistent kernel pays off once its scoring items fill the machine at least twice (its last items run after the
-    // pooling has ended); smaller layers take the three kernels.
+    // The persistent kernel pays off once its scoring items fill the machine (its last items run after the pooling has
+    // ended); smaller layers take the three kernels.
     int sms = 0;
     st = sm_count(&sms);
     if (st != CARNATOR_OK) return st;
-    const bool fused_able = p->mode == CARNATOR_MODE_TOPK && nkb <= 32 * 32 && tma_strides_ok(s, s->q_stride) && tma_strides_ok(s, s->k_stride) &&
-                            fused_smem_bytes(s->D, nkb) <= kMaxDynamicSmem;
-    const bool fused_pays = int64_t(s->B) * s->H * ceil_div(nqb, kFusedRows) >= 2 * int64_t(sms);
     const int choice = g_builder_path.load();
+    const bool fused_able = p->mode == CARNATOR_MODE_TOPK && nkb <= 32 * 32 && tma_strides_ok(s, s->q_stride) && tma_strides_ok(s, s->k_stride) &&
+                            fused_fits(s->D, nkb);
+    const bool fused_pays = int64_t(s->B) * s->H * ceil_div(nqb, kFusedRows) >= int64_t(sms);
     if (fused_able && (choice == 2 || (choice == 0 && fused_pays))) {
         // one persistent kernel: pooling, pooled scores and selection; the scores stay on chip
         FusedArgs fa;
@@ -240,12 +240,12 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
         fa.B = s->B; fa.scale = effective_scale(s);
         fa.nkb_pad = (nkb + 3) & ~3;
         CUtensorMap maps[4];     // Q, K: one box = 64 elements x one block of tokens (rows >= N read as zero); the three-term
-                                 // means of Q: 16 rows per box; of K: 128 rows per box
+                                 // means of Q: one item's rows per box; of K: 128 rows x 32 columns per box
         const int64_t bh = int64_t(s->B) * s->H;
         if (!tc::make_map(&maps[0], Q, s->B, s->H, s->N, s->D, s->q_stride, s->block_q) ||
             !tc::make_map(&maps[1], K, s->B, s->H, s->N, s->D, s->k_stride, s->block_k) ||
             !tc::make_map_2d(&maps[2], w.qsplit, 3 * bh * nqb, s->D, kFusedRows) ||
-            !tc::make_map_2d(&maps[3], w.ksplit, 3 * bh * nkb, s->D, 128)) {
+            !tc::make_map_2d(&maps[3], w.ksplit, 3 * bh * nkb, s->D, 128, 32)) {
             snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed or is unavailable");
             return CARNATOR_ERR_CUDA;
         }
