@@ -212,34 +212,42 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         // ================= pooling producer =================
         if (lane == 0) {
             tc::prefetch_tmap(&mapQ); tc::prefetch_tmap(&mapK);
-            // item number -> tensor-map coordinates; K blocks of a head first, then its Q blocks
-            auto coords = [&](int item, int& which, int& I, int& h, int& b) {
-                const int bh = item / per_head, rem = item - bh * per_head;
-                which = rem < nkb ? 1 : 0;
-                I = which ? rem : rem - nkb;
-                b = bh / H; h = bh - b * H;
-                return bh;
+            // Item number -> (head, block): a head's K blocks first, then its Q blocks.  This thread is the pooling path's
+            // serial part (a block every 0.7 us at full rate), so an item number is divided only once per batch of four
+            // and stepped from there.
+            struct Dec { int bh, rem, h, b; };
+            auto decode = [&](int item) {
+                Dec d; d.bh = item / per_head; d.rem = item - d.bh * per_head; d.b = d.bh / H; d.h = d.bh - d.b * H; return d;
             };
+            auto advance = [&](Dec& d) {
+                if (++d.rem == per_head) { d.rem = 0; ++d.bh; if (++d.h == H) { d.h = 0; ++d.b; } }
+            };
+            const int blk_q = a.pool.block[0], blk_k = a.pool.block[1];
+            const int64_t tstride_q = int64_t(heads) * nqb * D, tstride_k = int64_t(heads) * nkb * D;
+            __nv_bfloat16* const split_q = a.split[0];
+            __nv_bfloat16* const split_k = a.split[1];
             // Items are taken four at a time (one counter update per four blocks; consecutive blocks also sit next to
             // each other in HBM).  While one batch is loaded, L2 is asked for the whole next batch.
-            auto prefetch_batch = [&](int base) {
-                for (int j = 0; j < kFusedBatch; ++j) {
-                    if (base + j >= pool_total) break;
-                    int which, I, h, b; coords(base + j, which, I, h, b);
-                    const int block = which ? a.pool.block[1] : a.pool.block[0];
+            auto prefetch_batch = [&](int base, Dec d) {
+                for (int j = 0; j < kFusedBatch && base + j < pool_total; ++j, advance(d)) {
+                    const int which = d.rem < nkb ? 1 : 0;
+                    const int row0 = which ? d.rem * blk_k : (d.rem - nkb) * blk_q;
 #pragma unroll
-                    for (int x = 0; x < D / 64; ++x) tma_prefetch_4d(which ? &mapK : &mapQ, x * 64, I * block, h, b);
+                    for (int x = 0; x < D / 64; ++x) tma_prefetch_4d(which ? &mapK : &mapQ, x * 64, row0, d.h, d.b);
                 }
             };
             int base_cur = atomicAdd(&a.hdr->work[0], kFusedBatch);
             int base_next = atomicAdd(&a.hdr->work[0], kFusedBatch);
-            prefetch_batch(base_cur);
+            Dec dec_cur = decode(base_cur);
+            prefetch_batch(base_cur, dec_cur);
             int armed = -1, n = 0;
             bool more = true;
             while (more) {
-                prefetch_batch(base_next);
+                const Dec dec_next = decode(base_next);
+                prefetch_batch(base_next, dec_next);
                 const int base_after = atomicAdd(&a.hdr->work[0], kFusedBatch);      // needed one batch from now: its latency hides
-                for (int j = 0; j < kFusedBatch; ++j, ++n) {
+                Dec d = dec_cur;
+                for (int j = 0; j < kFusedBatch; ++j, ++n, advance(d)) {
                     const int item = base_cur + j;
                     const int s = n % kFusedStages;
                     PoolItem it; it.dst = nullptr; it.term_stride = 0; it.nvalid = 0; it.bh = -1; it.block = 0;
@@ -252,23 +260,23 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                         tc::mbar_arrive(bar_full(s));
                         more = false; break;
                     }
-                    int which, I, h, b;
-                    const int bh = coords(item, which, I, h, b);
-                    const int block = which ? a.pool.block[1] : a.pool.block[0];
+                    const int which = d.rem < nkb ? 1 : 0;
+                    const int I = which ? d.rem : d.rem - nkb;
+                    const int block = which ? blk_k : blk_q;
                     const int nb = which ? nkb : nqb;
-                    it.dst = (which ? a.split[1] : a.split[0]) + (int64_t(bh) * nb + I) * D;
-                    it.term_stride = int64_t(heads) * nb * D;
+                    it.dst = (which ? split_k : split_q) + (int64_t(d.bh) * nb + I) * D;
+                    it.term_stride = which ? tstride_k : tstride_q;
                     it.nvalid = min(block, a.pool.N - I * block);
-                    it.bh = bh; it.block = block;
+                    it.bh = d.bh; it.block = block;
                     pool_q[n % kFusedQueue] = it;                      // read by the others only after bar_full / bar_acc of this item
                     tc::mbar_expect_tx(bar_full(s), uint32_t(block) * D * 2);
 #pragma unroll
                     for (int x = 0; x < D / 64; ++x)
                         tc::tma_load_4d(smem_base + uint32_t(L::kOffRing + s * L::kSlot + x * L::kBox), which ? &mapK : &mapQ,
-                                        bar_full(s), x * 64, I * block, h, b);
+                                        bar_full(s), x * 64, I * block, d.h, d.b);
                     armed = n;
                 }
-                base_cur = base_next; base_next = base_after;
+                base_cur = base_next; base_next = base_after; dec_cur = dec_next;
             }
             if (*abortp)       // copies in flight must land before the CTA gives its shared memory back
                 for (int k = 0; k < kFusedStages && armed - k >= 0; ++k)
