@@ -758,6 +758,26 @@ inline bool make_map(CUtensorMap* map, const void* base, int B, int H, int N, in
     return r == CUDA_SUCCESS;
 }
 
+// The same tensor with the head dimension split into its 64-element halves as a dimension of its own, behind the
+// tokens: one box = D/64 halves x box_rows tokens x 64 elements lands in shared memory as [half][token][64] (each
+// half a 128-byte-swizzled slab), so one copy fetches what make_map's boxes fetch in D/64.
+inline bool make_map_halves(CUtensorMap* map, const void* base, int B, int H, int N, int D, const int64_t st[3], int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[5] = {64, cuuint64_t(N), cuuint64_t(D / 64), cuuint64_t(H), cuuint64_t(B)};
+    const cuuint64_t row = cuuint64_t(st[2]) * 2;
+    if ((H > 1 && st[1] <= 0) || (B > 1 && st[0] <= 0)) return false;
+    const cuuint64_t s_h = st[1] > 0 ? cuuint64_t(st[1]) * 2 : row * N;
+    const cuuint64_t s_b = st[0] > 0 ? cuuint64_t(st[0]) * 2 : s_h * H;
+    cuuint64_t strides[4] = {row, 128, s_h, s_b};
+    cuuint32_t box[5] = {64, cuuint32_t(box_rows), cuuint32_t(D / 64), 1, 1};
+    cuuint32_t estr[5] = {1, 1, 1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // 2-D map over a row-major [rows, D] bf16 array: box = box_cols x box_rows (64 columns: 128-byte swizzle, 32 columns:
 // 64-byte swizzle), rows past the end read as zero.
 inline bool make_map_2d(CUtensorMap* map, const void* base, int64_t rows, int D, int box_rows, int box_cols = 64) {

@@ -66,9 +66,14 @@ __device__ __forceinline__ int ld_acquire(const int32_t* p) {
     asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
 }
-__device__ __forceinline__ void tma_prefetch_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
-                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+__device__ __forceinline__ void tma_prefetch_5d(const CUtensorMap* map, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile("cp.async.bulk.prefetch.tensor.5d.L2.global.tile [%0, {%1, %2, %3, %4, %5}];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
+        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
     asm volatile(
@@ -232,8 +237,7 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 for (int j = 0; j < kFusedBatch && base + j < pool_total; ++j, advance(d)) {
                     const int which = d.rem < nkb ? 1 : 0;
                     const int row0 = which ? d.rem * blk_k : (d.rem - nkb) * blk_q;
-#pragma unroll
-                    for (int x = 0; x < D / 64; ++x) tma_prefetch_4d(which ? &mapK : &mapQ, x * 64, row0, d.h, d.b);
+                    tma_prefetch_5d(which ? &mapK : &mapQ, 0, row0, 0, d.h, d.b);
                 }
             };
             int base_cur = atomicAdd(&a.hdr->work[0], kFusedBatch);
@@ -270,10 +274,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     it.bh = d.bh; it.block = block;
                     pool_q[n % kFusedQueue] = it;                      // read by the others only after bar_full / bar_acc of this item
                     tc::mbar_expect_tx(bar_full(s), uint32_t(block) * D * 2);
-#pragma unroll
-                    for (int x = 0; x < D / 64; ++x)
-                        tc::tma_load_4d(smem_base + uint32_t(L::kOffRing + s * L::kSlot + x * L::kBox), which ? &mapK : &mapQ,
-                                        bar_full(s), x * 64, I * block, d.h, d.b);
+                    tma_load_5d(smem_base + uint32_t(L::kOffRing + s * L::kSlot), which ? &mapK : &mapQ, bar_full(s),
+                                0, I * block, 0, d.h, d.b);               // both halves of the head dimension in one copy
                     armed = n;
                 }
                 base_cur = base_next; base_next = base_after; dec_cur = dec_next;
@@ -285,10 +287,9 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     } else if (warp_id == 5) {
         // ================= pooling sums on the tensor cores =================
         if (lane == 0) {
-            // A = the block, MN-major (rows = head-dimension elements, 64-element chunks one box apart; for D = 64 the
+            // A = the block, MN-major (rows = head-dimension elements, 64-element halves one behind the other; for D = 64 the
             // upper 64 rows of the 128-row product repeat the lower ones and are never read); B = ones, K-major.
             constexpr uint32_t idesc = tc::instr_desc(128, 16, 0) | (1u << 15);
-            const uint64_t da0 = tc::smem_desc(smem_base + uint32_t(L::kOffRing), D == 128 ? uint32_t(L::kBox) : 0u, 1024);
             const uint64_t db = tc::smem_desc(smem_base + uint32_t(L::kOffOnes), 16, 1024);
             bool ok = true;
             for (int n = 0; ok; ++n) {
@@ -303,7 +304,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 if (it.dst == nullptr) { tc::mbar_arrive(bar_acc(buf)); break; }      // pass the end marker on
                 tc::tc_fence_after();
                 const int ksteps = (it.block + 15) / 16;                              // token rows past the valid ones read as zero
-                const uint64_t da = da0 + uint64_t((uint32_t(s) * uint32_t(L::kSlot)) >> 4);
+                // the second 64-element half of the head dimension lies one block of 128-byte rows behind the first
+                const uint64_t da = tc::smem_desc(smem_base + uint32_t(L::kOffRing + s * L::kSlot), D == 128 ? uint32_t(it.block) * 128u : 0u, 1024);
                 for (int kk = 0; kk < ksteps; ++kk)
                     tc::mma_ss(tmem + uint32_t(buf * 16), da + uint64_t(kk * (2048 >> 4)), db, idesc, kk > 0 ? 1u : 0u);
                 tc::tc_commit(bar_acc(buf));
