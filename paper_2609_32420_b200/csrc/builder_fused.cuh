@@ -552,21 +552,32 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 if (c >= n_admit) { T = cand; exact = (c == n_admit); }
             }
             const bool any = n_admit > 0;                               // n_admit == 0: nothing is admitted by score
-            int gt = 0;
+            if (exact) {
+                // The search ended on a threshold that exactly n_admit keys reach (or nothing is admitted): every key
+                // at or above it is kept and no tie has to be broken.  Keys of always-kept and absent blocks are 0 < T.
 #pragma unroll
-            for (int q = 0; q < NPL; ++q) gt += (key[q] > T) ? 1 : 0;
-            gt = __reduce_add_sync(0xffffffffu, gt);
-            const int need_eq = n_admit - gt;                           // blocks with key == T, lowest block index first
-            int seen_eq = 0;
+                for (int q = 0; q < NPL; ++q) {
+                    const int J = q * 32 + lane;
+                    const bool keep = ((forced_bits[q >> 5] >> (q & 31)) & 1u) || (any && key[q] >= T);
+                    if (J < nkb) a.sel.mask[row + J] = keep ? 1 : 0;
+                }
+            } else {
+                int gt = 0;
 #pragma unroll
-            for (int q = 0; q < NPL; ++q) {
-                const int J = q * 32 + lane;
-                const bool eq = any && key[q] == T;
-                const unsigned bal = __ballot_sync(0xffffffffu, eq);
-                const int rank = seen_eq + __popc(bal & ((1u << lane) - 1u));
-                seen_eq += __popc(bal);
-                const bool keep = ((forced_bits[q >> 5] >> (q & 31)) & 1u) || (any && key[q] > T) || (eq && rank < need_eq);
-                if (J < nkb) a.sel.mask[row + J] = keep ? 1 : 0;
+                for (int q = 0; q < NPL; ++q) gt += (key[q] > T) ? 1 : 0;
+                gt = __reduce_add_sync(0xffffffffu, gt);
+                const int need_eq = n_admit - gt;                       // blocks with key == T, lowest block index first
+                int seen_eq = 0;
+#pragma unroll
+                for (int q = 0; q < NPL; ++q) {
+                    const int J = q * 32 + lane;
+                    const bool eq = key[q] == T;
+                    const unsigned bal = __ballot_sync(0xffffffffu, eq);
+                    const int rank = seen_eq + __popc(bal & ((1u << lane) - 1u));
+                    seen_eq += __popc(bal);
+                    const bool keep = ((forced_bits[q >> 5] >> (q & 31)) & 1u) || key[q] > T || (eq && rank < need_eq);
+                    if (J < nkb) a.sel.mask[row + J] = keep ? 1 : 0;
+                }
             }
         }
         named_bar(2, NT);                                              // the rows are free for the next pass / item
