@@ -52,10 +52,10 @@ struct FusedArgs {
     int nkb_pad;            // row stride of the shared-memory score rows (floats)
 };
 
-struct PoolItem {           // one decoded pooling item, producer -> epilogue
-    __nv_bfloat16* dst;     // first of the three terms' rows (nullptr: end marker); the others follow term_stride apart
-    int64_t term_stride;
-    int nvalid, bh, block;  // valid tokens, head, token rows of the tile
+struct __align__(16) PoolItem {   // one pooling item, producer -> MMA warp and epilogue (16 bytes: one shared-memory store)
+    int bh;                 // head (batch-major); < 0: end marker
+    int I;                  // block index, bit 30 set for a K block
+    int block, nvalid;      // token rows of the tile, valid tokens among them
 };
 struct ScoreItem { int bh, I0; };     // bh < 0: end marker
 
@@ -188,7 +188,11 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             ok = tc::mbar_wait_warp(bar_acc(buf), uint32_t(n >> 1) & 1u, abortp, 64);
             if (!ok) { if (lane == 0 && !*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 41, n, blockIdx.x); break; }
             const PoolItem it = pool_q[n % kFusedQueue];
-            if (it.dst == nullptr) break;                              // the producer's end marker
+            if (it.bh < 0) break;                                      // the producer's end marker
+            // where the three terms go (this warp has time to spare; the producer thread does not)
+            const int which = it.I >> 30, I = it.I & 0x3FFFFFFF, nb = which ? nkb : nqb;
+            __nv_bfloat16* const dst = a.split[which] + (int64_t(it.bh) * nb + I) * D;
+            const int64_t term_stride = int64_t(heads) * nb * D;
             tc::tc_fence_after();
             const float sum = tmem_ld1(tmem + lane_base + uint32_t(buf * 16));
             tc::tmem_wait_ld();
@@ -200,7 +204,7 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 const float r1 = m - __bfloat162float(t1);
                 const __nv_bfloat16 t2 = __float2bfloat16_rn(r1);
                 const __nv_bfloat16 t3 = __float2bfloat16_rn(r1 - __bfloat162float(t2));
-                it.dst[d] = t1; it.dst[it.term_stride + d] = t2; it.dst[2 * it.term_stride + d] = t3;
+                dst[d] = t1; dst[term_stride + d] = t2; dst[2 * term_stride + d] = t3;
             }
             // A head's counter moves when this CTA leaves the head (one fence per head, not one per block).  The named
             // barrier orders the four warps' stores before thread 0's fence.
@@ -228,9 +232,6 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 if (++d.rem == per_head) { d.rem = 0; ++d.bh; if (++d.h == H) { d.h = 0; ++d.b; } }
             };
             const int blk_q = a.pool.block[0], blk_k = a.pool.block[1];
-            const int64_t tstride_q = int64_t(heads) * nqb * D, tstride_k = int64_t(heads) * nkb * D;
-            __nv_bfloat16* const split_q = a.split[0];
-            __nv_bfloat16* const split_k = a.split[1];
             // Items are taken four at a time (one counter update per four blocks; consecutive blocks also sit next to
             // each other in HBM).  While one batch is loaded, L2 is asked for the whole next batch.
             auto prefetch_batch = [&](int base, Dec d) {
@@ -254,7 +255,7 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 for (int j = 0; j < kFusedBatch; ++j, ++n, advance(d)) {
                     const int item = base_cur + j;
                     const int s = n % kFusedStages;
-                    PoolItem it; it.dst = nullptr; it.term_stride = 0; it.nvalid = 0; it.bh = -1; it.block = 0;
+                    PoolItem it; it.bh = -1; it.I = 0; it.block = 0; it.nvalid = 0;
                     if (n >= kFusedStages && !tc::mbar_wait(bar_empty(s), uint32_t(n / kFusedStages - 1) & 1u, abortp, 64)) {
                         if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 42, n, blockIdx.x);
                         *abortp = 1; more = false; break;
@@ -267,11 +268,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     const int which = d.rem < nkb ? 1 : 0;
                     const int I = which ? d.rem : d.rem - nkb;
                     const int block = which ? blk_k : blk_q;
-                    const int nb = which ? nkb : nqb;
-                    it.dst = (which ? split_k : split_q) + (int64_t(d.bh) * nb + I) * D;
-                    it.term_stride = which ? tstride_k : tstride_q;
+                    it.bh = d.bh; it.I = I | (which << 30); it.block = block;
                     it.nvalid = min(block, a.pool.N - I * block);
-                    it.bh = d.bh; it.block = block;
                     pool_q[n % kFusedQueue] = it;                      // read by the others only after bar_full / bar_acc of this item
                     tc::mbar_expect_tx(bar_full(s), uint32_t(block) * D * 2);
                     tma_load_5d(smem_base + uint32_t(L::kOffRing + s * L::kSlot), which ? &mapK : &mapQ, bar_full(s),
@@ -301,7 +299,7 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     ok = tc::mbar_wait(bar_accfree(buf), uint32_t((n - 2) >> 1) & 1u, abortp, 32);
                     if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 44, n, blockIdx.x); *abortp = 1; break; }
                 }
-                if (it.dst == nullptr) { tc::mbar_arrive(bar_acc(buf)); break; }      // pass the end marker on
+                if (it.bh < 0) { tc::mbar_arrive(bar_acc(buf)); break; }              // pass the end marker on
                 tc::tc_fence_after();
                 const int ksteps = (it.block + 15) / 16;                              // token rows past the valid ones read as zero
                 // the second 64-element half of the head dimension lies one block of 128-byte rows behind the first
