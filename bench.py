@@ -456,7 +456,7 @@ def dense_lse(D, w, inputs):
 
 
 def leg_seed_expansion(D, w, inputs, n):
-    """carnator_seed_expansion: reads Q once (the seed keys are a few hundred rows), so HBM bandwidth bounds it."""
+    """carnator_seed_expansion: Q is read once and multiplied by a few hundred gathered key rows per head."""
     torch, cn = D.torch, D.cn
     Qh, Kh = inputs["Qh"], inputs["Kh"]
     Lh = dense_lse(D, w, inputs)
@@ -465,15 +465,17 @@ def leg_seed_expansion(D, w, inputs, n):
     tok = rng.choice(np.arange(w.n_text, w.N), size=n_pos + n_neg, replace=False).astype(np.int32)
     seeds = torch.from_numpy(tok).to(D.dev)
     shape = cn.shape_of(w, Qh, Kh)
-    ms, ms_min, clocks = D.timed(lambda: cn.seed_expansion(Qh, Kh, Lh, seeds, n_pos, n_neg, shape), n)
+    ws = torch.empty(cn.seed_workspace_bytes(shape), dtype=torch.uint8, device=D.dev)
+    ms, ms_min, clocks = D.timed(lambda: cn.seed_expansion(Qh, Kh, Lh, seeds, n_pos, n_neg, shape, ws=ws), n)
+    status = cn.query_status(ws)
     nbytes = float(w.B) * w.H * w.N * (w.D * 2 + 4 + 4) + float(w.B) * w.N * 4     # Q, LSE, per-head contrast, result
     flops = 2.0 * w.B * w.H * w.N * (n_pos + n_neg) * w.D                          # Q x K_seed^T
     return {"ms": ms, "ms_min": ms_min, "n_pos": n_pos, "n_neg": n_neg, "bytes_per_launch": nbytes, "flops_per_launch": flops,
             "gbs": nbytes / (ms * 1e-3) / 1e9, "frac_of_hbm": nbytes / (ms * 1e-3) / 1e9 / D.peaks["hbm"],
             "tflops": flops / (ms * 1e-3) / 1e12, "frac_of_bf16_burst": flops / (ms * 1e-3) / 1e12 / D.peaks["bf16"],
-            "bound": "tensor (mma.sync) at this seed count; hbm (read Q once) below about 100 seeds",
-            "executor": "mma.sync (Q x K_seed^T on gathered key rows)", "clocks": clocks,
-            "note": "includes the allocation of its workspace and output by the binding"}
+            "bound": "tensor at this seed count; hbm (read Q once) below about 100 seeds",
+            "executor": "tcgen05 (Q tile x 256 gathered seed key rows per product; gather kernel and head mean included)",
+            "status": status, "clocks": clocks}
 
 
 def leg_regions(D, w, inputs, n):

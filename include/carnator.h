@@ -292,7 +292,13 @@ carnator_status carnator_sparse_attn_region(const void* Q, const void* K, const 
  *             heads and batch entries; an empty set contributes 0
  *   per_head_opt  device, fp32 [B,H,N] or NULL: the per-head contrasts
  *   contrast  device, fp32 [B,N], written
- *   ws        device workspace, 256-byte aligned, >= carnator_seed_workspace_bytes
+ *   ws        device workspace, 256-byte aligned, >= carnator_seed_workspace_bytes (status header, the
+ *             per-head contrasts, and the seed tokens' key rows gathered per head: 512 rows)
+ *
+ * Up to 512 seeds in all (and a query tensor that is not shared over heads or batch entries) run on the
+ * tcgen05 tensor cores: a gather kernel, a persistent product-and-maximum kernel with bounded waits whose
+ * status carnator_query_status(ws) returns, and the mean over heads.  Larger seed sets run on an mma.sync
+ * kernel that streams the seed rows in chunks of 64.  A seed index outside [0, N) counts as a zero key row.
  * ------------------------------------------------------------------------ */
 size_t carnator_seed_workspace_bytes(const carnator_shape* shape);
 

@@ -436,15 +436,22 @@ def sparse_attn_region(Q, K, V, mask, active_q, context_k, shape: Shape, O, LSE,
     return ws
 
 
-def seed_expansion(Q, K, LSE, seeds, n_pos: int, n_neg: int, shape: Shape, per_head=None, stream=None):
-    """carnator_seed_expansion.  seeds: int32 device tensor [n_pos + n_neg].  Returns contrast fp32 [B,N]."""
+def seed_workspace_bytes(shape: Shape) -> int:
+    return int(lib().carnator_seed_workspace_bytes(ctypes.byref(shape)))
+
+
+def seed_expansion(Q, K, LSE, seeds, n_pos: int, n_neg: int, shape: Shape, per_head=None, stream=None, ws=None,
+                   return_ws: bool = False):
+    """carnator_seed_expansion.  seeds: int32 device tensor [n_pos + n_neg].  Returns contrast fp32 [B,N]
+    (and the workspace, whose header carries the device status, with ``return_ws``)."""
     import torch
     out = torch.empty((shape.B, shape.N), dtype=torch.float32, device=Q.device)
-    ws = _new_ws(int(lib().carnator_seed_workspace_bytes(ctypes.byref(shape))), Q.device)
+    if ws is None:
+        ws = _new_ws(int(lib().carnator_seed_workspace_bytes(ctypes.byref(shape))), Q.device)
     st = lib().carnator_seed_expansion(_ptr(Q), _ptr(K), _ptr(LSE), _ptr(seeds), n_pos, n_neg, ctypes.byref(shape),
                                        _ptr(per_head), _ptr(out), _ptr(ws), ws.numel(), _stream(stream))
     _check(st, "carnator_seed_expansion")
-    return out
+    return (out, ws) if return_ws else out
 
 
 # ---- host-side scalars (no GPU) ---------------------------------------------------------------------

@@ -16,6 +16,7 @@
 #include "block_mass_tcgen05.cuh"
 #include "regions.cuh"
 #include "seed_expand.cuh"
+#include "seed_expand_tcgen05.cuh"
 #include "compat_host.inl"
 
 using namespace carnator;
@@ -798,7 +799,8 @@ extern "C" carnator_status carnator_sparse_attn_region(const void* Q, const void
 // ------------------------------------------------------------------------------------------------
 extern "C" size_t carnator_seed_workspace_bytes(const carnator_shape* s) {
     if (check_shape(s, false) != CARNATOR_OK) return 0;
-    return align256(sizeof(WsHeader)) + align256(size_t(s->B) * s->H * s->N * 4);
+    // header | per-head contrasts [B,H,N] fp32 | gathered seed key rows [B,H,512,D] bf16
+    return align256(sizeof(WsHeader)) + align256(size_t(s->B) * s->H * s->N * 4) + align256(seed_gather_bytes(s));
 }
 
 extern "C" carnator_status carnator_seed_expansion(const void* Q, const void* K, const float* LSE, const int32_t* seeds,
@@ -821,6 +823,37 @@ extern "C" carnator_status carnator_seed_expansion(const void* Q, const void* K,
     a.per_head = per_head_opt ? per_head_opt : reinterpret_cast<float*>(static_cast<char*>(ws) + align256(sizeof(WsHeader)));
     a.B = s->B; a.H = s->H; a.N = s->N;
     a.scale_log2 = effective_scale(s) * kLog2e;
+    const int64_t n_bn = int64_t(s->B) * s->N;
+    if (seed_tcgen05_supported(s, n_pos + n_neg)) {
+        WsHeader* hdr = static_cast<WsHeader*>(ws);
+        CUDA_TRY(cudaMemsetAsync(hdr, 0, sizeof(WsHeader), stream));
+        int sms = 0;
+        st = sm_count(&sms);
+        if (st != CARNATOR_OK) return st;
+        tc::SeedGatherArgs ga;
+        ga.K = a.K; for (int i = 0; i < 3; ++i) ga.ks[i] = a.ks[i];
+        ga.seeds = seeds; ga.n_seeds = n_pos + n_neg; ga.H = s->H; ga.N = s->N;
+        ga.out = reinterpret_cast<__nv_bfloat16*>(static_cast<char*>(ws) + align256(sizeof(WsHeader)) +
+                                                   align256(size_t(s->B) * s->H * s->N * 4));
+        tc::SeedTcArgs ta;
+        ta.LSE = LSE; ta.per_head = a.per_head; ta.hdr = hdr;
+        ta.n_pos = n_pos; ta.n_seeds = n_pos + n_neg;
+        ta.B = s->B; ta.H = s->H; ta.N = s->N; ta.nqb = ceil_div(s->N, tc::kBlock);
+        ta.tiles = s->B * s->H * ta.nqb;
+        ta.scale_log2 = a.scale_log2;
+        CUtensorMap mq, ms;      // the gathered rows as one [B*H*512, D] array: a box = 256 seed rows x 64 elements
+        if (!tc::make_map(&mq, Q, s->B, s->H, s->N, s->D, s->q_stride, tc::kBlock) ||
+            !tc::make_map_2d(&ms, ga.out, int64_t(s->B) * s->H * tc::kSeedCap, s->D, tc::kSeedChunk)) {
+            snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed or is unavailable");
+            return CARNATOR_ERR_CUDA;
+        }
+        st = s->D == 128 ? launch_seed_tc<128>(ga, ta, mq, ms, sms, stream, g_cuda_error, sizeof(g_cuda_error))
+                         : launch_seed_tc<64>(ga, ta, mq, ms, sms, stream, g_cuda_error, sizeof(g_cuda_error));
+        if (st != CARNATOR_OK) return st;
+        head_mean_kernel<<<unsigned((n_bn + 255) / 256), 256, 0, stream>>>(a.per_head, s->B, s->H, s->N, contrast);
+        LAUNCH_CHECK("head_mean_kernel");
+        return CARNATOR_OK;
+    }
     dim3 grid(ceil_div(s->N, 128), s->H, s->B);
     if (s->D == 128) {
         const size_t smem = size_t(128 + 2 * 64) * (128 + 8) * 2;

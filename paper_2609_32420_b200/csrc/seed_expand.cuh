@@ -2,8 +2,9 @@
 //   S_i = mean_h [ max_{u in I+} A_h[i,u] - max_{u in I-} A_h[i,u] ],   A_h[i,u] = exp(s_iu - LSE_i),
 // with I+ / I- the noun and background seed token sets (Section 3.2, evidence region construction;
 // Appendix "Evidence Region Construction").  exp is monotone, so per head only the largest score over each
-// seed set is needed: a Q x K_seed^T product on gathered key rows (mma.sync, the seed sets are small) followed
-// by row maxima, then one exponential per query, head and set.
+// seed set is needed: a Q x K_seed^T product on gathered key rows followed by row maxima, then one exponential
+// per query, head and set.  This file holds the mma.sync form, which streams the seed rows in chunks of 64 and takes
+// any number of them; calls with at most 512 seeds run on the tcgen05 kernel of seed_expand_tcgen05.cuh instead.
 #pragma once
 #include "attn_portable.cuh"
 

@@ -16,6 +16,11 @@ pytestmark = pytest.mark.gpu
     ("wan1p3b_480p", dict(H=3, T=3), 150, 333),      # ragged seed counts (not multiples of 64), ragged N
     ("cogvideox5b", dict(H=2, T=2), 64, 1),          # D = 64, text tokens present
     ("wan1p3b_480p", dict(H=1, T=2), 5, 0),          # empty background set
+    ("wan1p3b_480p", dict(H=1, T=2), 0, 40),         # empty noun set
+    ("wan1p3b_480p", dict(H=3, T=8), 192, 320),      # 512 seeds: both tensor-memory chunks full; CTAs whose tile range spans two heads
+    ("wan1p3b_480p", dict(H=2, T=3), 300, 100),      # the set boundary falls inside a chunk and inside a group of 32 columns
+    ("cogvideox5b", dict(H=5, T=6), 257, 255),       # D = 64, a boundary one past the first chunk
+    ("wan1p3b_480p", dict(H=2, T=2), 400, 200),      # more seeds than the tensor-core form takes: the mma.sync kernel
 ])
 def test_seed_expansion_matches_oracle(name, kw, n_pos, n_neg):
     w = wl.shrunk(wl.get(name), **kw)
@@ -30,7 +35,9 @@ def test_seed_expansion_matches_oracle(name, kw, n_pos, n_neg):
     tok = rng.choice(np.arange(w.n_text, w.N), size=n_pos + n_neg, replace=False).astype(np.int32)
     seeds = torch.from_numpy(tok).cuda()
     per_head = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device="cuda")
-    out = cn.seed_expansion(Q, K, L, seeds, n_pos, n_neg, cn.shape_of(w, Q, K), per_head=per_head)
+    out, sws = cn.seed_expansion(Q, K, L, seeds, n_pos, n_neg, cn.shape_of(w, Q, K), per_head=per_head, return_ws=True)
+    if 0 < n_pos + n_neg <= 512:
+        assert cn.query_status(sws) == cn.OK, cn.last_cuda_error()
     S_ref, ph_ref = orc.seed_expansion(Qb, Kb, w.N, w.scale, tok[:n_pos], tok[n_pos:])
     for got, ref in ((per_head.cpu().numpy(), ph_ref), (out.cpu().numpy(), S_ref)):
         assert (np.abs(got - ref) <= 1e-3 * np.abs(ref) + 2e-6).all(), float(np.abs(got - ref).max())
