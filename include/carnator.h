@@ -108,7 +108,8 @@ typedef struct carnator_build_params {
  *          receives S (and replaces the score area of the workspace)
  *   ws     device workspace, 256-byte aligned, >= carnator_build_workspace_bytes
  * In top-k mode with nkb <= 1024, on layers large enough to fill the GPU, the three steps run as one persistent
- * kernel (block sums on the tensor cores at HBM speed, fp32 scores and selection on chip beside them); otherwise,
+ * kernel (block sums and pooled scores on the tensor cores -- the means split into three bf16 terms, fp32 accumulate --
+ * at HBM speed, selection on chip beside them); otherwise,
  * and in cumulative-mass mode, as three kernels with the scores held in the workspace.
  * Limits: nkb <= 4096.
  * ------------------------------------------------------------------------ */
