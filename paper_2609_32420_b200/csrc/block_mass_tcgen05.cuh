@@ -47,7 +47,7 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     extern __shared__ unsigned char smem_dyn[];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
-    __shared__ float red[2][4][4];          // [group][slot][lane quarter] partial sums of one (I,J) tile
+    __shared__ float red[2][8][4];          // [group][slot][lane quarter] partial sums of one (I,J) tile
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int b = blockIdx.z, h = blockIdx.y, I = blockIdx.x;
@@ -65,7 +65,7 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
     auto bar_kempty = [&](int s) { return bars + 64 + 8 * s; };
     auto bar_sfull = [&](int s) { return bars + 96 + 8 * s; };
     auto bar_sfree = [&](int s) { return bars + 128 + 8 * s; };
-    auto bar_red = [&](int g, int s) { return bars + 160 + 8 * (g * 4 + s); };
+    auto bar_red = [&](int g, int s) { return bars + 160 + 8 * (g * 8 + s); };
     volatile int* abortp = &abort_flag;
 
     if (tid == 0) {
@@ -74,7 +74,7 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
         for (int s = 0; s < kMassStages; ++s) { mbar_init(bar_kfull(s), 1); mbar_init(bar_kempty(s), 1); }
         for (int s = 0; s < kMassSBufs; ++s) { mbar_init(bar_sfull(s), 1); mbar_init(bar_sfree(s), 4); }
         for (int g = 0; g < 2; ++g)
-            for (int s = 0; s < 4; ++s) mbar_init(bar_red(g, s), 4);
+            for (int s = 0; s < 8; ++s) mbar_init(bar_red(g, s), 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == kMassWarpTma && lane == 0) { prefetch_tmap(&mapQ); prefetch_tmap(&mapK); }
@@ -166,28 +166,62 @@ block_mass_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constan
             tmem_wait_ld();
             tc_fence_before();
             mbar_arrive_warp(bar_sfree(sb));     // the scores are in registers: the buffer may be refilled
-            const float neg = -lse2;             // -inf for rows past N: exp2(-inf) = 0
-            float part[4] = {0.f, 0.f, 0.f, 0.f};
+            // exp2(s * scale - lse2), two scores per FMA-pipe instruction; -inf offset for rows past N gives 0
+            float v;
+            if (nvalid == kBlock) {
+                const uint64_t neg2 = pack2(-lse2, -lse2), scale2 = pack2(a.scale_log2, a.scale_log2);
+                uint64_t part2[4] = {pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
+                for (int c = 0; c < 4; ++c)
 #pragma unroll
-                for (int e = 0; e < 32; ++e) {
-                    const float p = ex2_approx(fmaf(s[c][e], a.scale_log2, neg));
-                    part[e & 3] += (c * 32 + e < nvalid) ? p : 0.f;     // keys >= N never count
-                }
-            float v = (part[0] + part[1]) + (part[2] + part[3]);
+                    for (int e = 0; e < 16; ++e) {
+                        float x0, x1;
+                        unpack2(fma2(pack2(s[c][2 * e], s[c][2 * e + 1]), scale2, neg2), x0, x1);
+                        part2[e & 3] = add2(part2[e & 3], pack2(ex2_approx(x0), ex2_approx(x1)));
+                    }
+                float p0, p1, p2, p3, p4, p5, p6, p7;
+                unpack2(part2[0], p0, p1); unpack2(part2[1], p2, p3); unpack2(part2[2], p4, p5); unpack2(part2[3], p6, p7);
+                v = ((p0 + p1) + (p2 + p3)) + ((p4 + p5) + (p6 + p7));
+            } else {                              // the ragged last key block (warp-uniform): keys >= N never count
+                const float neg = -lse2;
+                float part[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) {
+                        const float p = ex2_approx(fmaf(s[c][e], a.scale_log2, neg));
+                        part[e & 3] += (c * 32 + e < nvalid) ? p : 0.f;
+                    }
+                v = (part[0] + part[1]) + (part[2] + part[3]);
+            }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-            // four warps of the group -> one value; the first warp adds them in a fixed order
-            const int slot = (i >> 1) & 3;
-            if (lane == 0) red[wg][slot][quarter] = v;
-            mbar_arrive_warp(bar_red(wg, slot));
-            if (quarter == 0) {
-                ok = mbar_wait_warp(bar_red(wg, slot), uint32_t(i >> 3) & 1u, abortp, 0);
+            // Four warps of the group -> one value; the first warp adds them in a fixed order.  It does so two of the
+            // group's tiles later, when the other warps' arrivals are long past, so nobody stops for the hand-over
+            // (eight slots per group: a warp can be two tiles ahead of the slowest warp of its group, no more, because
+            // a score buffer is refilled only when all four have read it; a slot is rewritten eight tiles on).
+            const int n = i >> 1;                       // this group's n-th tile
+            if (lane == 0) red[wg][n & 7][quarter] = v;
+            mbar_arrive_warp(bar_red(wg, n & 7));
+            if (quarter == 0 && n >= 2) {
+                const int m = n - 2;
+                ok = mbar_wait_warp(bar_red(wg, m & 7), uint32_t(m >> 3) & 1u, abortp, 0);
                 if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 37, i, blockIdx.x); break; }
                 if (lane == 0) {
-                    const float tot = ((red[wg][slot][0] + red[wg][slot][1]) + red[wg][slot][2]) + red[wg][slot][3];
-                    a.mass[(bh * a.nqb + I) * int64_t(a.nkb) + i] = tot * inv_rows;
+                    const float tot = ((red[wg][m & 7][0] + red[wg][m & 7][1]) + red[wg][m & 7][2]) + red[wg][m & 7][3];
+                    a.mass[(bh * a.nqb + I) * int64_t(a.nkb) + (2 * m + wg)] = tot * inv_rows;
+                }
+            }
+        }
+        // the group's last two tiles
+        if (quarter == 0 && ok) {
+            const int ntile = (T - wg + 1) / 2;         // tiles this group has handled
+            for (int m = max(0, ntile - 2); m < ntile && ok; ++m) {
+                ok = mbar_wait_warp(bar_red(wg, m & 7), uint32_t(m >> 3) & 1u, abortp, 0);
+                if (!ok) { if (lane == 0) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 37, m, blockIdx.x); break; }
+                if (lane == 0) {
+                    const float tot = ((red[wg][m & 7][0] + red[wg][m & 7][1]) + red[wg][m & 7][2]) + red[wg][m & 7][3];
+                    a.mass[(bh * a.nqb + I) * int64_t(a.nkb) + (2 * m + wg)] = tot * inv_rows;
                 }
             }
         }
