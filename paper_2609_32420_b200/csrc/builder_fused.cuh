@@ -33,11 +33,12 @@ namespace carnator {
 constexpr int kFusedPoolThreads = 256;      // warps 0-7: pooling (0-5) and score operands / products (6-7)
 constexpr int kFusedScoreThreads = 512;     // warps 8-23: selection group
 constexpr int kFusedThreads = kFusedPoolThreads + kFusedScoreThreads;
-constexpr int kFusedStages = 3;       // blocks in the pooling ring
-constexpr int kFusedBatch = 4;        // pooling items taken per counter update; L2 is asked for one batch ahead
-constexpr int kFusedQueue = 8;        // decoded items in flight between producer and epilogue (> kFusedStages + 2)
+// blocks in the pooling ring (PST: 3, or 2 where the score rows of a long layer need the room) and buffers of the
+// key-block operand of the score products (AST: 3 where they fit, else 2) are template parameters of the kernel
+constexpr int kFusedBatchBytes = 64 * 1024;    // consecutive bytes of Q or K a CTA takes per counter update (2 or 4 blocks)
+constexpr int kFusedAheadBytes = 128 * 1024;   // how far ahead of the loads L2 is asked for the blocks to come
+constexpr int kFusedQueue = 8;        // decoded items in flight between producer and epilogue (> PST + 2)
 constexpr int kFusedRows = 16;        // query blocks per scoring item (N of the score products; one selection warp each)
-constexpr int kFusedAStages = 2;      // buffers of the key-block operand of the score products
 constexpr int kFusedTmemCols = 512;   // [0, 32): two pooling accumulators; [32, 512): score tiles
 
 struct FusedArgs {
@@ -100,15 +101,15 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 // Score operands: A = the three terms of 128 key-block means, one 32-element quarter of the head dimension at a time
 // (3 boxes of 128 rows x 64 B, 64-byte swizzle), two buffers; B = the three terms of the item's 16 query-block means,
 // whole rows (boxes of 16 rows x 128 B, 128-byte swizzle).
-template <int D>
+template <int D, int PST, int AST>
 struct FusedSmem {
     static constexpr size_t kBox = size_t(128) * 128;
     static constexpr size_t kBoxB = size_t(kFusedRows) * 128;                     // 16 query blocks x 64 elements
     static constexpr size_t kSlot = (D / 64) * kBox;
     static constexpr size_t kOffRing = 0;                                         // 1 KiB aligned
     static constexpr size_t kBoxA = size_t(128) * 64;                             // 128 key blocks x 32 elements, 64-byte swizzle
-    static constexpr size_t kOffScoreA = kOffRing + kFusedStages * kSlot;         // kFusedAStages buffers x 3 terms x 8 KiB
-    static constexpr size_t kOffScoreB = kOffScoreA + kFusedAStages * 3 * kBoxA;  // 3 terms x D/64 halves x 2 KiB
+    static constexpr size_t kOffScoreA = kOffRing + PST * kSlot;                  // AST buffers x 3 terms x 8 KiB
+    static constexpr size_t kOffScoreB = kOffScoreA + AST * 3 * kBoxA;            // 3 terms x D/64 halves x 2 KiB
     static constexpr size_t kOffOnes = kOffScoreB + 3 * (D / 64) * kBoxB;         // 16 rows x 128 B of bf16 ones
     static constexpr size_t kOffBar = kOffOnes + 2048;                            // mbarriers
     static constexpr size_t kOffScores = kOffBar + 256;                           // float [RP][nkb_pad]
@@ -116,17 +117,19 @@ struct FusedSmem {
     static size_t bytes(int nkb, int nkb_pad) { return off_scores(nkb) + size_t(kFusedRows) * nkb_pad * 4 + 1024; }   // + slack to align the base
 };
 
-template <int D, int NPL>
+template <int D, int NPL, int PST, int AST>
 __global__ void __launch_bounds__(kFusedThreads, 1)
 build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapK,
                    const __grid_constant__ CUtensorMap mapQs, const __grid_constant__ CUtensorMap mapKs, const FusedArgs a) {
     extern __shared__ unsigned char fsm_raw[];
     __shared__ PoolItem pool_q[kFusedQueue];
+    __shared__ int ahead_q[8 * 5];                      // the pooling producer's batches taken from the counter and not yet loaded
     __shared__ ScoreItem score_q[4];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     constexpr int NR = kFusedRows, RP = kFusedRows;                 // query blocks per item = rows selected at once
-    using L = FusedSmem<D>;
+    constexpr int kBatch = kFusedBatchBytes / (128 * D * 2);           // pooling items per counter update: 2 (D = 128) or 4
+    using L = FusedSmem<D, PST, AST>;
     constexpr int KH = D / 64;                                         // 64-element halves of the head dimension
     // accumulators per score tile: the large product t1 t1, one per half of the head dimension, apart from the five small ones
     constexpr int NACC = KH + 1;
@@ -150,10 +153,10 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
 
     if (tid == 0) {
         abort_flag = 0;
-        for (int s = 0; s < kFusedStages; ++s) { tc::mbar_init(bar_full(s), 1); tc::mbar_init(bar_empty(s), 1); }
+        for (int s = 0; s < PST; ++s) { tc::mbar_init(bar_full(s), 1); tc::mbar_init(bar_empty(s), 1); }
         for (int s = 0; s < 2; ++s) { tc::mbar_init(bar_acc(s), 1); tc::mbar_init(bar_accfree(s), 4); }
         tc::mbar_init(bar_drain, 1); tc::mbar_init(bar_drain2, 1);
-        for (int s = 0; s < kFusedAStages; ++s) { tc::mbar_init(bar_afull(s), 1); tc::mbar_init(bar_afree(s), 1); }
+        for (int s = 0; s < AST; ++s) { tc::mbar_init(bar_afull(s), 1); tc::mbar_init(bar_afree(s), 1); }
         tc::mbar_init(bar_bfull, 1); tc::mbar_init(bar_bfree, 1);
         tc::mbar_init(bar_sfull, 1); tc::mbar_init(bar_sfree, kFusedScoreThreads / 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -206,8 +209,9 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 const __nv_bfloat16 t3 = __float2bfloat16_rn(r1 - __bfloat162float(t2));
                 dst[d] = t1; dst[term_stride + d] = t2; dst[2 * term_stride + d] = t3;
             }
-            // A head's counter moves when this CTA leaves the head (one fence per head, not one per block).  The named
-            // barrier orders the four warps' stores before thread 0's fence.
+            // A head's counter moves when this CTA leaves the head (one fence per head, not one per block: a fence per
+            // batch of two blocks slowed the whole kernel by a fifth).  The named barrier orders the four warps' stores
+            // before thread 0's fence.
             named_bar(1, 128);
             if (tid == 0) {
                 if (it.bh != pub_head && pub_count > 0) { __threadfence(); atomicAdd(&a.done[pub_head], pub_count); pub_count = 0; }
@@ -222,41 +226,45 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
         if (lane == 0) {
             tc::prefetch_tmap(&mapQ); tc::prefetch_tmap(&mapK);
             // Item number -> (head, block): a head's K blocks first, then its Q blocks.  This thread is the pooling path's
-            // serial part (a block every 0.7 us at full rate), so an item number is divided only once per batch of four
-            // and stepped from there.
-            struct Dec { int bh, rem, h, b; };
+            // serial part (a block every 0.7 us at full rate), so an item number is divided only once per batch and
+            // stepped from there.
+            struct Dec { int base, bh, rem, h, b; };
             auto decode = [&](int item) {
-                Dec d; d.bh = item / per_head; d.rem = item - d.bh * per_head; d.b = d.bh / H; d.h = d.bh - d.b * H; return d;
+                Dec d; d.base = item; d.bh = item / per_head; d.rem = item - d.bh * per_head; d.b = d.bh / H; d.h = d.bh - d.b * H; return d;
             };
             auto advance = [&](Dec& d) {
                 if (++d.rem == per_head) { d.rem = 0; ++d.bh; if (++d.h == H) { d.h = 0; ++d.b; } }
             };
             const int blk_q = a.pool.block[0], blk_k = a.pool.block[1];
-            // Items are taken four at a time (one counter update per four blocks; consecutive blocks also sit next to
-            // each other in HBM).  While one batch is loaded, L2 is asked for the whole next batch.
-            auto prefetch_batch = [&](int base, Dec d) {
-                for (int j = 0; j < kFusedBatch && base + j < pool_total; ++j, advance(d)) {
+            // Items are taken two at a time from the counter (small batches keep the CTAs level and a head's counter
+            // moving), but L2 is asked for them 128 KB ahead of the loads: the batches taken and not yet loaded wait,
+            // decoded, in a small queue.
+            auto prefetch_batch = [&](Dec d) {
+                for (int j = 0; j < kBatch && d.base + j < pool_total; ++j, advance(d)) {
                     const int which = d.rem < nkb ? 1 : 0;
                     const int row0 = which ? d.rem * blk_k : (d.rem - nkb) * blk_q;
                     tma_prefetch_5d(which ? &mapK : &mapQ, 0, row0, 0, d.h, d.b);
                 }
             };
-            int base_cur = atomicAdd(&a.hdr->work[0], kFusedBatch);
-            int base_next = atomicAdd(&a.hdr->work[0], kFusedBatch);
-            Dec dec_cur = decode(base_cur);
-            prefetch_batch(base_cur, dec_cur);
+            constexpr int kAhead = kFusedAheadBytes / int(L::kSlot) / kBatch;     // batches between counter and load
+            static_assert(kAhead >= 1 && kAhead < 8, "look-ahead queue");
+            Dec* const ahead = reinterpret_cast<Dec*>(ahead_q);
+            for (int k = 0; k < kAhead; ++k) { ahead[k] = decode(atomicAdd(&a.hdr->work[0], kBatch)); prefetch_batch(ahead[k]); }
+            int pending = atomicAdd(&a.hdr->work[0], kBatch);       // its value is needed one batch from now: the latency hides
             int armed = -1, n = 0;
             bool more = true;
-            while (more) {
-                const Dec dec_next = decode(base_next);
-                prefetch_batch(base_next, dec_next);
-                const int base_after = atomicAdd(&a.hdr->work[0], kFusedBatch);      // needed one batch from now: its latency hides
-                Dec d = dec_cur;
-                for (int j = 0; j < kFusedBatch; ++j, ++n, advance(d)) {
+            for (int nb = 0; more; ++nb) {
+                const Dec fresh = decode(pending);
+                ahead[(nb + kAhead) & 7] = fresh;
+                prefetch_batch(fresh);
+                pending = atomicAdd(&a.hdr->work[0], kBatch);
+                Dec d = ahead[nb & 7];
+                const int base_cur = d.base;
+                for (int j = 0; j < kBatch; ++j, ++n, advance(d)) {
                     const int item = base_cur + j;
-                    const int s = n % kFusedStages;
+                    const int s = n % PST;
                     PoolItem it; it.bh = -1; it.I = 0; it.block = 0; it.nvalid = 0;
-                    if (n >= kFusedStages && !tc::mbar_wait(bar_empty(s), uint32_t(n / kFusedStages - 1) & 1u, abortp, 64)) {
+                    if (n >= PST && !tc::mbar_wait(bar_empty(s), uint32_t(n / PST - 1) & 1u, abortp, 64)) {
                         if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 42, n, blockIdx.x);
                         *abortp = 1; more = false; break;
                     }
@@ -276,11 +284,10 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                                 0, I * block, 0, d.h, d.b);               // both halves of the head dimension in one copy
                     armed = n;
                 }
-                base_cur = base_next; base_next = base_after; dec_cur = dec_next;
             }
             if (*abortp)       // copies in flight must land before the CTA gives its shared memory back
-                for (int k = 0; k < kFusedStages && armed - k >= 0; ++k)
-                    tc::mbar_wait_drain(bar_full((armed - k) % kFusedStages), uint32_t((armed - k) / kFusedStages) & 1u);
+                for (int k = 0; k < PST && armed - k >= 0; ++k)
+                    tc::mbar_wait_drain(bar_full((armed - k) % PST), uint32_t((armed - k) / PST) & 1u);
         }
     } else if (warp_id == 5) {
         // ================= pooling sums on the tensor cores =================
@@ -291,8 +298,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const uint64_t db = tc::smem_desc(smem_base + uint32_t(L::kOffOnes), 16, 1024);
             bool ok = true;
             for (int n = 0; ok; ++n) {
-                const int s = n % kFusedStages, buf = n & 1;
-                ok = tc::mbar_wait(bar_full(s), uint32_t(n / kFusedStages) & 1u, abortp, 32);
+                const int s = n % PST, buf = n & 1;
+                ok = tc::mbar_wait(bar_full(s), uint32_t(n / PST) & 1u, abortp, 32);
                 if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 43, n, blockIdx.x); *abortp = 1; break; }
                 const PoolItem it = pool_q[n % kFusedQueue];
                 if (n >= 2) {
@@ -352,9 +359,9 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                                     kh * 64, t3 * rows_q + si.bh * nqb + si.I0);
                 for (int t = 0; t < ntiles && ok; ++t)
                     for (int kq = 0; kq < 2 * KH; ++kq, ++step) {        // quarters of 32 elements, the buffers in turn
-                        const int buf = step % kFusedAStages;
-                        if (step >= kFusedAStages) {
-                            ok = tc::mbar_wait(bar_afree(buf), uint32_t(step / kFusedAStages - 1) & 1u, abortp, 32);
+                        const int buf = step % AST;
+                        if (step >= AST) {
+                            ok = tc::mbar_wait(bar_afree(buf), uint32_t(step / AST - 1) & 1u, abortp, 32);
                             if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 46, step, blockIdx.x); *abortp = 1; break; }
                         }
                         tc::mbar_expect_tx(bar_afull(buf), uint32_t(3 * L::kBoxA));
@@ -365,8 +372,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             }
             // on the way out after an abort, copies in flight must land first; an unarmed barrier simply runs out
             if (*abortp)
-                for (int k = 1; k <= kFusedAStages && step - k >= 0; ++k)
-                    tc::mbar_wait_drain(bar_afull((step - k) % kFusedAStages), uint32_t((step - k) / kFusedAStages) & 1u, 20000000ull);
+                for (int k = 1; k <= AST && step - k >= 0; ++k)
+                    tc::mbar_wait_drain(bar_afull((step - k) % AST), uint32_t((step - k) / AST) & 1u, 20000000ull);
         }
     } else if (warp_id == 7) {
         // ================= scores on the tensor cores =================
@@ -390,8 +397,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 if (si.bh < 0) { tc::mbar_arrive(bar_sfull); break; }                   // pass the end marker on
                 for (int t = 0; t < ntiles && ok; ++t)
                     for (int kq = 0; kq < 2 * KH; ++kq, ++step) {
-                        const int buf = step % kFusedAStages, kh = kq >> 1;
-                        ok = tc::mbar_wait(bar_afull(buf), uint32_t(step / kFusedAStages) & 1u, abortp, 32);
+                        const int buf = step % AST, kh = kq >> 1;
+                        ok = tc::mbar_wait(bar_afull(buf), uint32_t(step / AST) & 1u, abortp, 32);
                         if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 49, step, blockIdx.x); *abortp = 1; break; }
                         tc::tc_fence_after();
                         // The tensor cores add into an fp32 accumulator without guard bits, so a long chain of additions

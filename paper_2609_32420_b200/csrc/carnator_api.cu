@@ -135,34 +135,54 @@ carnator_status sm_count(int* out) {
 
 constexpr size_t kMaxDynamicSmem = 226 * 1024;     // 227 KiB per CTA less the kernels' static shared memory
 
-template <int D, int NPL>
+template <int D, int NPL, int PST, int AST>
 carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap (&maps)[4], int nkb, int sms, cudaStream_t stream) {
-    const size_t smem = FusedSmem<D>::bytes(nkb, fa.nkb_pad);
-    carnator_status st = allow_smem(build_fused_kernel<D, NPL>, smem);
+    const size_t smem = FusedSmem<D, PST, AST>::bytes(nkb, fa.nkb_pad);
+    carnator_status st = allow_smem(build_fused_kernel<D, NPL, PST, AST>, smem);
     if (st != CARNATOR_OK) return st;
     // the register hand-over inside the kernel (setmaxnreg) only completes if the CTA owns 256 x 40 + 512 x 96 registers
     cudaFuncAttributes attr;
-    CUDA_TRY(cudaFuncGetAttributes(&attr, build_fused_kernel<D, NPL>));
+    CUDA_TRY(cudaFuncGetAttributes(&attr, build_fused_kernel<D, NPL, PST, AST>));
     if (attr.numRegs * kFusedThreads < 256 * 40 + 512 * 96) {
         snprintf(g_cuda_error, sizeof(g_cuda_error), "build_fused_kernel was built with %d registers per thread: too few for its setmaxnreg split", attr.numRegs);
         return CARNATOR_ERR_UNSUPPORTED;
     }
-    build_fused_kernel<D, NPL><<<sms, kFusedThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], fa);
+    build_fused_kernel<D, NPL, PST, AST><<<sms, kFusedThreads, smem, stream>>>(maps[0], maps[1], maps[2], maps[3], fa);
     LAUNCH_CHECK("build_fused_kernel");
     return CARNATOR_OK;
 }
 
-bool fused_fits(int D, int nkb) {
+// Shared-memory plan of the fused kernel: pooling ring slots x buffers of the key-block score operand.  Three and three
+// where the score rows (which grow with the number of key blocks) leave the room; a long layer gives up a ring slot
+// rather than the third operand buffer (its scoring, not its pooling, is what the kernel waits for); else three and two.
+// 0: nothing fits.
+template <int D>
+int fused_plan_d(int nkb) {
     const int pad = (nkb + 3) & ~3;
-    return (D == 128 ? FusedSmem<128>::bytes(nkb, pad) : FusedSmem<64>::bytes(nkb, pad)) <= kMaxDynamicSmem;
+    if (FusedSmem<D, 3, 3>::bytes(nkb, pad) <= kMaxDynamicSmem) return 33;
+    if (FusedSmem<D, 2, 3>::bytes(nkb, pad) <= kMaxDynamicSmem) return 23;
+    if (FusedSmem<D, 3, 2>::bytes(nkb, pad) <= kMaxDynamicSmem) return 32;
+    return 0;
 }
+int fused_plan(int D, int nkb) { return D == 128 ? fused_plan_d<128>(nkb) : fused_plan_d<64>(nkb); }
+bool fused_fits(int D, int nkb) { return fused_plan(D, nkb) != 0; }
 
 // a warp of the selection group keeps the NPL keys of its row in registers
+template <int D, int NPL>
+carnator_status launch_fused_p(const FusedArgs& fa, const CUtensorMap (&maps)[4], int nkb, int sms, cudaStream_t stream) {
+    switch (fused_plan_d<D>(nkb)) {
+        case 33: return launch_fused_r<D, NPL, 3, 3>(fa, maps, nkb, sms, stream);
+        case 23: return launch_fused_r<D, NPL, 2, 3>(fa, maps, nkb, sms, stream);
+        case 32: return launch_fused_r<D, NPL, 3, 2>(fa, maps, nkb, sms, stream);
+        default: return CARNATOR_ERR_UNSUPPORTED;
+    }
+}
+
 template <int D>
 carnator_status launch_fused_d(const FusedArgs& fa, const CUtensorMap (&maps)[4], int nkb, int sms, cudaStream_t stream) {
-    if (nkb <= 32 * 8) return launch_fused_r<D, 8>(fa, maps, nkb, sms, stream);
-    if (nkb <= 32 * 20) return launch_fused_r<D, 20>(fa, maps, nkb, sms, stream);
-    return launch_fused_r<D, 32>(fa, maps, nkb, sms, stream);
+    if (nkb <= 32 * 8) return launch_fused_p<D, 8>(fa, maps, nkb, sms, stream);
+    if (nkb <= 32 * 20) return launch_fused_p<D, 20>(fa, maps, nkb, sms, stream);
+    return launch_fused_p<D, 32>(fa, maps, nkb, sms, stream);
 }
 
 carnator_status launch_fused_builder(const FusedArgs& fa, const CUtensorMap (&maps)[4], int D, int nkb, int sms, cudaStream_t stream) {
