@@ -55,7 +55,7 @@ struct FusedArgs {
 
 struct __align__(16) PoolItem {   // one pooling item, producer -> MMA warp and epilogue (16 bytes: one shared-memory store)
     int bh;                 // head (batch-major); < 0: end marker
-    int I;                  // block index, bit 30 set for a K block
+    int I;                  // (first) block index, bit 30 set for a K block
     int block, nvalid;      // token rows of the tile, valid tokens among them
 };
 struct ScoreItem { int bh, I0; };     // bh < 0: end marker
@@ -105,7 +105,7 @@ template <int D, int PST, int AST>
 struct FusedSmem {
     static constexpr size_t kBox = size_t(128) * 128;
     static constexpr size_t kBoxB = size_t(kFusedRows) * 128;                     // 16 query blocks x 64 elements
-    static constexpr size_t kSlot = (D / 64) * kBox;
+    static constexpr size_t kSlot = 2 * kBox;                                    // D = 128: the two halves of a block; D = 64: two blocks
     static constexpr size_t kOffRing = 0;                                         // 1 KiB aligned
     static constexpr size_t kBoxA = size_t(128) * 64;                             // 128 key blocks x 32 elements, 64-byte swizzle
     static constexpr size_t kOffScoreA = kOffRing + PST * kSlot;                  // AST buffers x 3 terms x 8 KiB
@@ -128,7 +128,10 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
     constexpr int NR = kFusedRows, RP = kFusedRows;                 // query blocks per item = rows selected at once
-    constexpr int kBatch = kFusedBatchBytes / (128 * D * 2);           // pooling items per counter update: 2 (D = 128) or 4
+    constexpr int kBatch = kFusedBatchBytes / int(FusedSmem<D, PST, AST>::kSlot);   // pooling items per counter update (2)
+    // A pooling item fills the 128 rows of the tensor-core product: at D = 128 one block (its two 64-element halves), at
+    // D = 64 two consecutive blocks of the same tensor and head.
+    constexpr int PB = D == 64 ? 2 : 1;
     using L = FusedSmem<D, PST, AST>;
     constexpr int KH = D / 64;                                         // 64-element halves of the head dimension
     // accumulators per score tile: the large product t1 t1, one per half of the head dimension, apart from the five small ones
@@ -172,7 +175,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     tc::tc_fence_after();
     const uint32_t tmem = tmem_slot;
     const uint32_t tmem_s = tmem + 32;                                // score tiles (behind the two pooling accumulators)
-    const int per_head = nqb + nkb;
+    const int nqi = (nqb + PB - 1) / PB, nki = (nkb + PB - 1) / PB;     // pooling items per head and tensor
+    const int per_head = nqi + nki;
     const int pool_total = heads * per_head;
     const int groups_per_head = (nqb + NR - 1) / NR;
     const int score_total = heads * groups_per_head;
@@ -182,7 +186,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     if (warp_id < 8) asm volatile("setmaxnreg.dec.sync.aligned.u32 40;" ::: "memory");
     if (warp_id < 4) {
         // ================= pooling epilogue: tensor memory -> block means as three bf16 terms =================
-        const int d = warp_id * 32 + lane;                             // head-dimension element = tensor-memory lane
+        const int r = warp_id * 32 + lane;                             // tensor-memory lane: head-dimension element (and block, D = 64)
+        const int d = r & (D - 1);
         const uint32_t lane_base = uint32_t(warp_id * 32) << 16;
         int pub_count = 0, pub_head = -1;
         bool ok = true;
@@ -193,7 +198,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             const PoolItem it = pool_q[n % kFusedQueue];
             if (it.bh < 0) break;                                      // the producer's end marker
             // where the three terms go (this warp has time to spare; the producer thread does not)
-            const int which = it.I >> 30, I = it.I & 0x3FFFFFFF, nb = which ? nkb : nqb;
+            const int which = it.I >> 30, nb = which ? nkb : nqb;
+            const int I = (it.I & 0x3FFFFFFF) + r / D;                  // this lane's block (D = 64: lanes 64-127 hold the item's second block)
             __nv_bfloat16* const dst = a.split[which] + (int64_t(it.bh) * nb + I) * D;
             const int64_t term_stride = int64_t(heads) * nb * D;
             tc::tc_fence_after();
@@ -201,8 +207,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             tc::tmem_wait_ld();
             tc::tc_fence_before();
             tc::mbar_arrive_warp(bar_accfree(buf));
-            if (d < D) {
-                const float m = sum / float(it.nvalid);
+            if (I < nb) {
+                const float m = sum / float(min(it.block, a.pool.N - I * it.block));
                 const __nv_bfloat16 t1 = __float2bfloat16_rn(m);
                 const float r1 = m - __bfloat162float(t1);
                 const __nv_bfloat16 t2 = __float2bfloat16_rn(r1);
@@ -241,8 +247,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             // decoded, in a small queue.
             auto prefetch_batch = [&](Dec d) {
                 for (int j = 0; j < kBatch && d.base + j < pool_total; ++j, advance(d)) {
-                    const int which = d.rem < nkb ? 1 : 0;
-                    const int row0 = which ? d.rem * blk_k : (d.rem - nkb) * blk_q;
+                    const int which = d.rem < nki ? 1 : 0;
+                    const int row0 = which ? d.rem * PB * blk_k : (d.rem - nki) * PB * blk_q;
                     tma_prefetch_5d(which ? &mapK : &mapQ, 0, row0, 0, d.h, d.b);
                 }
             };
@@ -273,15 +279,15 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                         tc::mbar_arrive(bar_full(s));
                         more = false; break;
                     }
-                    const int which = d.rem < nkb ? 1 : 0;
-                    const int I = which ? d.rem : d.rem - nkb;
+                    const int which = d.rem < nki ? 1 : 0;
+                    const int I = (which ? d.rem : d.rem - nki) * PB;      // the item's first block
                     const int block = which ? blk_k : blk_q;
                     it.bh = d.bh; it.I = I | (which << 30); it.block = block;
                     it.nvalid = min(block, a.pool.N - I * block);
                     pool_q[n % kFusedQueue] = it;                      // read by the others only after bar_full / bar_acc of this item
-                    tc::mbar_expect_tx(bar_full(s), uint32_t(block) * D * 2);
+                    tc::mbar_expect_tx(bar_full(s), uint32_t(PB * block) * D * 2);     // rows past N arrive as zeros and count
                     tma_load_5d(smem_base + uint32_t(L::kOffRing + s * L::kSlot), which ? &mapK : &mapQ, bar_full(s),
-                                0, I * block, 0, d.h, d.b);               // both halves of the head dimension in one copy
+                                0, I * block, 0, d.h, d.b);               // both halves of the head dimension, or both blocks, in one copy
                     armed = n;
                 }
             }
@@ -292,8 +298,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
     } else if (warp_id == 5) {
         // ================= pooling sums on the tensor cores =================
         if (lane == 0) {
-            // A = the block, MN-major (rows = head-dimension elements, 64-element halves one behind the other; for D = 64 the
-            // upper 64 rows of the 128-row product repeat the lower ones and are never read); B = ones, K-major.
+            // A = the item, MN-major: rows = head-dimension elements, the second 64 rows one block of 128-byte rows behind
+            // the first (D = 128: the second half of the head dimension; D = 64: the next block); B = ones, K-major.
             constexpr uint32_t idesc = tc::instr_desc(128, 16, 0) | (1u << 15);
             const uint64_t db = tc::smem_desc(smem_base + uint32_t(L::kOffOnes), 16, 1024);
             bool ok = true;
@@ -309,8 +315,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                 if (it.bh < 0) { tc::mbar_arrive(bar_acc(buf)); break; }              // pass the end marker on
                 tc::tc_fence_after();
                 const int ksteps = (it.block + 15) / 16;                              // token rows past the valid ones read as zero
-                // the second 64-element half of the head dimension lies one block of 128-byte rows behind the first
-                const uint64_t da = tc::smem_desc(smem_base + uint32_t(L::kOffRing + s * L::kSlot), D == 128 ? uint32_t(it.block) * 128u : 0u, 1024);
+                // rows 64-127 of the operand lie one block of 128-byte rows behind rows 0-63
+                const uint64_t da = tc::smem_desc(smem_base + uint32_t(L::kOffRing + s * L::kSlot), uint32_t(it.block) * 128u, 1024);
                 for (int kk = 0; kk < ksteps; ++kk)
                     tc::mma_ss(tmem + uint32_t(buf * 16), da + uint64_t(kk * (2048 >> 4)), db, idesc, kk > 0 ? 1u : 0u);
                 tc::tc_commit(bar_acc(buf));

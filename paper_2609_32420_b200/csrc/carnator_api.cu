@@ -263,8 +263,9 @@ extern "C" carnator_status carnator_build_connectivity(const void* Q, const void
         CUtensorMap maps[4];     // Q, K: one box = one block of tokens, all of D (rows >= N read as zero); the three-term
                                  // means of Q: one item's rows per box; of K: 128 rows x 32 columns per box
         const int64_t bh = int64_t(s->B) * s->H;
-        if (!tc::make_map_halves(&maps[0], Q, s->B, s->H, s->N, s->D, s->q_stride, s->block_q) ||
-            !tc::make_map_halves(&maps[1], K, s->B, s->H, s->N, s->D, s->k_stride, s->block_k) ||
+        const int pb = s->D == 64 ? 2 : 1;       // at D = 64 a pooling item is two consecutive blocks (one box)
+        if (!tc::make_map_halves(&maps[0], Q, s->B, s->H, s->N, s->D, s->q_stride, pb * s->block_q) ||
+            !tc::make_map_halves(&maps[1], K, s->B, s->H, s->N, s->D, s->k_stride, pb * s->block_k) ||
             !tc::make_map_2d(&maps[2], w.qsplit, 3 * bh * nqb, s->D, kFusedRows) ||
             !tc::make_map_2d(&maps[3], w.ksplit, 3 * bh * nkb, s->D, 128, 32)) {
             snprintf(g_cuda_error, sizeof(g_cuda_error), "cuTensorMapEncodeTiled failed or is unavailable");
