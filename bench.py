@@ -434,12 +434,24 @@ def leg_exact_builder(D, w, inputs, n):
     ms, ms_min, clocks = D.timed(lambda: cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, ws=xws), n)
     x_flops = 2.0 * w.B * w.H * float(w.N) * float(w.N) * w.D
     tiles = w.B * w.H * w.nqb * w.nkb
+    # How the pooled-score estimator's mask (the one the timed steps run under) relates to the exact block masses of the
+    # same history pair: reported, not a pass / fail (the paper prints no mask to compare with).
+    bm = torch.empty((w.B, w.H, w.nqb, w.nkb), dtype=torch.float32, device=D.dev)
+    cn.build_connectivity_exact(Qh, Kh, Lh, bshape, xparams, mask=xmask, block_mass=bm, ws=xws)
+    est = inputs["mask"] != 0
+    exact = xmask != 0
+    fidelity = {"estimator_mask_density": float(est.float().mean()),
+                "attention_mass_under_estimator_mask": float((bm * est).sum(-1).mean()),
+                "attention_mass_under_exact_mask": float((bm * exact).sum(-1).mean()),
+                "estimator_recall_of_exact_mask": float((est & exact).sum() / exact.sum().clamp(min=1)),
+                "exact_mask_recall_of_estimator": float((est & exact).sum() / est.sum().clamp(min=1))}
+    del bm
     mufu = mufu_bound_ms(tiles, w.block, clocks.get("sm_mhz"))
     tf = x_flops / (ms * 1e-3) / 1e12
     return {"ms": ms, "ms_min": ms_min, "tflops": tf, "flops_per_launch": x_flops, "mass": w.build.mass,
             "density": float(xmask.float().mean()), "status": cn.query_status(xws),
             "bound": "exponential unit", "mufu_bound_ms": mufu, "frac_of_mufu_bound": (mufu / ms) if mufu else None,
-            "frac_of_bf16_burst": tf / D.peaks["bf16"], "clocks": clocks}
+            "frac_of_bf16_burst": tf / D.peaks["bf16"], "estimator_fidelity": fidelity, "clocks": clocks}
 
 
 def dense_lse(D, w, inputs):
