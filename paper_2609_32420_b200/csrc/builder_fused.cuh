@@ -99,7 +99,7 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 
 // Shared-memory plan.  Pooling ring: blocks of 128 token rows as D/64 boxes (128 rows x 128 B, 128-byte swizzle).
 // Score operands: A = the three terms of 128 key-block means, one 32-element quarter of the head dimension at a time
-// (3 boxes of 128 rows x 64 B, 64-byte swizzle), two buffers; B = the three terms of the item's 16 query-block means,
+// (3 boxes of 128 rows x 64 B, 64-byte swizzle), AST buffers; B = the three terms of the item's 16 query-block means,
 // whole rows (boxes of 16 rows x 128 B, 128-byte swizzle).
 template <int D, int PST, int AST>
 struct FusedSmem {
