@@ -8,7 +8,8 @@
 //               divides by the number of valid tokens and writes the block mean as three bf16 terms
 //               (mean = t1 + t2 + t3 to fp32 precision)
 //   warp 4      pooling producer (one lane): takes (head, tensor, block) items from a counter and brings each block
-//               into a shared-memory ring with TMA (and asks L2 for blocks further ahead)
+//               into a shared-memory ring with TMA (and asks L2 for blocks further ahead); at D = 64 an item is two
+//               consecutive blocks, which fill the 128 rows of the product as the two halves of a D = 128 block do
 //   warp 5      pooling sums on the tensor cores (one lane): sum over tokens = X^T (the block as an MN-major A
 //               operand, one row per head-dimension element) times a 128 x 16 matrix of ones, fp32 accumulate in
 //               tensor memory; the CUDA cores then only touch D values per block
