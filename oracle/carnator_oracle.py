@@ -470,27 +470,31 @@ def attention_region_rows(Qb, Kb, Vb, N, block_q, block_k, scale, mask, active_q
 # ==========================================================================
 # Seeded self-attention expansion (Section 3.2; Appendix "Evidence Region Construction")
 # ==========================================================================
-def seed_expansion(Qb, Kb, N, scale, seeds_pos, seeds_neg, lse: Optional[np.ndarray] = None):
+def seed_expansion(Qb, Kb, N, scale, seeds_pos, seeds_neg, lse: Optional[np.ndarray] = None,
+                   heads=None, rows: Optional[np.ndarray] = None):
     """S_i = mean_h [ max_{u in I+} A_h[i,u] - max_{u in I-} A_h[i,u] ] with A the dense self-attention
     weights (softmax over all N keys).  Returns (contrast [B, N], per_head [B, H, N]) in fp64.  ``lse``
     [B, H, N] may be supplied; otherwise the softmax normaliser is computed here.  An empty seed set
-    contributes 0."""
+    contributes 0.  With ``heads`` (a list of (b, h)) and / or ``rows`` (query token indices) only those
+    entries of per_head are computed (the others stay 0, and the contrast is then not meaningful): the
+    same arithmetic, for sampled checks of layers too large to do in full."""
     B, H = Qb.shape[0], Qb.shape[1]
     per_head = np.zeros((B, H, N))
     sp = np.asarray(seeds_pos, dtype=np.int64)
     sn = np.asarray(seeds_neg, dtype=np.int64)
-    for b in range(B):
-        for h in range(H):
-            q, k = _widen(Qb[b, h, :N]), _widen(Kb[b, h, :N])
-            if lse is None:
-                l = np.zeros(N)
-                for i0 in range(0, N, 1024):
-                    l[i0:i0 + 1024] = np.logaddexp.reduce(scale * (q[i0:i0 + 1024] @ k.T), axis=1)
-            else:
-                l = lse[b, h]
-            pos = np.exp(scale * (q @ k[sp].T) - l[:, None]).max(axis=1) if sp.size else 0.0
-            neg = np.exp(scale * (q @ k[sn].T) - l[:, None]).max(axis=1) if sn.size else 0.0
-            per_head[b, h] = pos - neg
+    sel = np.arange(N) if rows is None else np.asarray(rows, dtype=np.int64)
+    todo = [(b, h) for b in range(B) for h in range(H)] if heads is None else list(heads)
+    for (b, h) in todo:
+        q, k = _widen(Qb[b, h, :N])[sel], _widen(Kb[b, h, :N])
+        if lse is None:
+            l = np.zeros(len(sel))
+            for i0 in range(0, len(sel), 1024):
+                l[i0:i0 + 1024] = np.logaddexp.reduce(scale * (q[i0:i0 + 1024] @ k.T), axis=1)
+        else:
+            l = lse[b, h][sel]
+        pos = np.exp(scale * (q @ k[sp].T) - l[:, None]).max(axis=1) if sp.size else 0.0
+        neg = np.exp(scale * (q @ k[sn].T) - l[:, None]).max(axis=1) if sn.size else 0.0
+        per_head[b, h, sel] = pos - neg
     return per_head.mean(axis=1), per_head
 
 

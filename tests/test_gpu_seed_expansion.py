@@ -41,3 +41,37 @@ def test_seed_expansion_matches_oracle(name, kw, n_pos, n_neg):
     S_ref, ph_ref = orc.seed_expansion(Qb, Kb, w.N, w.scale, tok[:n_pos], tok[n_pos:])
     for got, ref in ((per_head.cpu().numpy(), ph_ref), (out.cpu().numpy(), S_ref)):
         assert (np.abs(got - ref) <= 1e-3 * np.abs(ref) + 2e-6).all(), float(np.abs(got - ref).max())
+
+
+def test_full_size_layer_on_sampled_rows():
+    """The Wan-14B-shaped layer in the launch configuration the bench times (one CTA per SM, about 160 query tiles
+    each, most CTAs crossing a head boundary); the oracle checks 384 query rows of three heads, with its own
+    softmax normaliser: every 128-row tile position, the ragged last tile and tiles next to head boundaries."""
+    import os
+    w = wl.get("wan14b_720p")
+    nthreads = min(16, os.cpu_count() or 1)
+    Qb, Kb = wl.gen_tensor(w, "Q", threads=nthreads), wl.gen_tensor(w, "K", threads=nthreads)
+    Q, K = to_dev(Qb), to_dev(Kb)
+    V = torch.zeros_like(Q)
+    shape = cn.shape_of(w, Q, K, V)
+    ones = torch.ones((w.B, w.H, w.nqb, w.nkb), dtype=torch.uint8, device="cuda")
+    _, L, ws = cn.sparse_attn(Q, K, V, ones, None, shape)
+    assert cn.query_status(ws) == cn.OK
+    del V, ones
+    n_pos, n_neg = 192, 320
+    rng = np.random.default_rng(7)
+    tok = rng.choice(np.arange(w.N), size=n_pos + n_neg, replace=False).astype(np.int32)
+    per_head = torch.empty((w.B, w.H, w.N), dtype=torch.float32, device="cuda")
+    out, sws = cn.seed_expansion(Q, K, L, torch.from_numpy(tok).cuda(), n_pos, n_neg, cn.shape_of(w, Q, K),
+                                 per_head=per_head, return_ws=True)
+    assert cn.query_status(sws) == cn.OK, cn.last_cuda_error()
+    heads = [(0, 0), (0, 17), (0, w.H - 1)]
+    rows = np.unique(np.concatenate([rng.choice(w.N, size=320, replace=False), np.arange(0, 40),
+                                     np.arange(w.N - 80, w.N), np.arange(128 * 300 - 8, 128 * 300 + 8)]))
+    _, ph_ref = orc.seed_expansion(Qb, Kb, w.N, w.scale, tok[:n_pos], tok[n_pos:], heads=heads, rows=rows)
+    got = per_head.cpu().numpy()
+    for (b, h) in heads:
+        g, r = got[b, h, rows], ph_ref[b, h, rows]
+        assert (np.abs(g - r) <= 1e-3 * np.abs(r) + 2e-6).all(), (h, float(np.abs(g - r).max()))
+    # the mean over heads is a plain reduction of per_head: check it against the GPU's own per-head values
+    np.testing.assert_allclose(out.cpu().numpy(), got.mean(axis=1), rtol=1e-5, atol=1e-7)

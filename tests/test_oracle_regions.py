@@ -122,3 +122,8 @@ def test_seed_expansion_matches_dense_softmax_matrix_and_invariants():
     assert (S_all >= 0).all()                                         # max over every key dominates any subset
     S_empty, ph = orc.seed_expansion(Q, K, N, 0.4, pos, [])
     assert (ph > 0).all()
+    # the sampled form (some heads, some query rows) gives the very entries of the full form and leaves the rest at 0
+    rows = np.array([1, 7, 8, 39])
+    _, ph_s = orc.seed_expansion(Q, K, N, 0.4, pos, neg, heads=[(0, 2), (0, 0)], rows=rows)
+    np.testing.assert_array_equal(ph_s[0, [0, 2]][:, rows], per_head[0, [0, 2]][:, rows])
+    assert (ph_s[0, 1] == 0).all() and (np.delete(ph_s[0, 0], rows) == 0).all()
