@@ -154,14 +154,12 @@ carnator_status launch_fused_r(const FusedArgs& fa, const CUtensorMap (&maps)[4]
 
 // Shared-memory plan of the fused kernel: pooling ring slots x buffers of the key-block score operand.  Three and three
 // where the score rows (which grow with the number of key blocks) leave the room; a long layer gives up a ring slot
-// rather than the third operand buffer (its scoring, not its pooling, is what the kernel waits for); else three and two.
-// 0: nothing fits.
+// rather than the third operand buffer (its scoring, not its pooling, is what the kernel waits for).  0: nothing fits.
 template <int D>
 int fused_plan_d(int nkb) {
     const int pad = (nkb + 3) & ~3;
     if (FusedSmem<D, 3, 3>::bytes(nkb, pad) <= kMaxDynamicSmem) return 33;
     if (FusedSmem<D, 2, 3>::bytes(nkb, pad) <= kMaxDynamicSmem) return 23;
-    if (FusedSmem<D, 3, 2>::bytes(nkb, pad) <= kMaxDynamicSmem) return 32;
     return 0;
 }
 int fused_plan(int D, int nkb) { return D == 128 ? fused_plan_d<128>(nkb) : fused_plan_d<64>(nkb); }
@@ -173,7 +171,6 @@ carnator_status launch_fused_p(const FusedArgs& fa, const CUtensorMap (&maps)[4]
     switch (fused_plan_d<D>(nkb)) {
         case 33: return launch_fused_r<D, NPL, 3, 3>(fa, maps, nkb, sms, stream);
         case 23: return launch_fused_r<D, NPL, 2, 3>(fa, maps, nkb, sms, stream);
-        case 32: return launch_fused_r<D, NPL, 3, 2>(fa, maps, nkb, sms, stream);
         default: return CARNATOR_ERR_UNSUPPORTED;
     }
 }
