@@ -61,6 +61,16 @@ struct __align__(16) PoolItem {   // one pooling item, producer -> MMA warp and 
 };
 struct ScoreItem { int bh, I0; };     // bh < 0: end marker
 
+// tcgen05.mma with both operands in shared memory, for a converged warp: every lane executes the statement with the same
+// operands and one elected lane issues (the compiler keeps the descriptors in uniform registers, and the warp spends far
+// fewer issue slots per instruction than a single lane inside a branch does)
+__device__ __forceinline__ void mma_ss_elect(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p, e;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+        "elect.sync _|e, 0xffffffff;\n\t"
+        "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void named_bar(int id, int nthreads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory"); }
 
 __device__ __forceinline__ int ld_acquire(const int32_t* p) {
@@ -297,8 +307,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     tc::mbar_wait_drain(bar_full((armed - k) % PST), uint32_t((armed - k) / PST) & 1u);
         }
     } else if (warp_id == 5) {
-        // ================= pooling sums on the tensor cores =================
-        if (lane == 0) {
+        // ================= pooling sums on the tensor cores (converged warp, one elected lane issues) =================
+        {
             // A = the item, MN-major: rows = head-dimension elements, the second 64 rows one block of 128-byte rows behind
             // the first (D = 128: the second half of the head dimension; D = 64: the next block); B = ones, K-major.
             constexpr uint32_t idesc = tc::instr_desc(128, 16, 0) | (1u << 15);
@@ -306,25 +316,26 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             bool ok = true;
             for (int n = 0; ok; ++n) {
                 const int s = n % PST, buf = n & 1;
-                ok = tc::mbar_wait(bar_full(s), uint32_t(n / PST) & 1u, abortp, 32);
-                if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 43, n, blockIdx.x); *abortp = 1; break; }
+                ok = tc::mbar_wait_warp(bar_full(s), uint32_t(n / PST) & 1u, abortp, 32);
+                if (!ok) { if (lane == 0) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 43, n, blockIdx.x); *abortp = 1; } break; }
                 const PoolItem it = pool_q[n % kFusedQueue];
                 if (n >= 2) {
-                    ok = tc::mbar_wait(bar_accfree(buf), uint32_t((n - 2) >> 1) & 1u, abortp, 32);
-                    if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 44, n, blockIdx.x); *abortp = 1; break; }
+                    ok = tc::mbar_wait_warp(bar_accfree(buf), uint32_t((n - 2) >> 1) & 1u, abortp, 32);
+                    if (!ok) { if (lane == 0) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 44, n, blockIdx.x); *abortp = 1; } break; }
                 }
-                if (it.bh < 0) { tc::mbar_arrive(bar_acc(buf)); break; }              // pass the end marker on
+                if (it.bh < 0) { if (lane == 0) tc::mbar_arrive(bar_acc(buf)); break; }              // pass the end marker on
                 tc::tc_fence_after();
                 const int ksteps = (it.block + 15) / 16;                              // token rows past the valid ones read as zero
                 // rows 64-127 of the operand lie one block of 128-byte rows behind rows 0-63
                 const uint64_t da = tc::smem_desc(smem_base + uint32_t(L::kOffRing + s * L::kSlot), uint32_t(it.block) * 128u, 1024);
                 for (int kk = 0; kk < ksteps; ++kk)
-                    tc::mma_ss(tmem + uint32_t(buf * 16), da + uint64_t(kk * (2048 >> 4)), db, idesc, kk > 0 ? 1u : 0u);
-                tc::tc_commit(bar_acc(buf));
-                tc::tc_commit(bar_empty(s));
+                    mma_ss_elect(tmem + uint32_t(buf * 16), da + uint64_t(kk * (2048 >> 4)), db, idesc, kk > 0 ? 1u : 0u);
+                tc::tc_commit_el(bar_acc(buf));
+                tc::tc_commit_el(bar_empty(s));
             }
-            tc::tc_commit(bar_drain);                                  // no product may still run when tensor memory is released
+            tc::tc_commit_el(bar_drain);                               // no product may still run when tensor memory is released
             tc::mbar_wait_drain(bar_drain, 0);
+            __syncwarp();
         }
     } else if (warp_id == 6) {
         // ================= score producer: the three-term means of an item's query blocks and of the head's key blocks =================
@@ -383,8 +394,8 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                     tc::mbar_wait_drain(bar_afull((step - k) % AST), uint32_t((step - k) / AST) & 1u, 20000000ull);
         }
     } else if (warp_id == 7) {
-        // ================= scores on the tensor cores =================
-        if (lane == 0) {
+        // ================= scores on the tensor cores (converged warp, one elected lane issues) =================
+        {
             // S^T tile t (128 key blocks x 16 query blocks) += A_term x B_term^T over the six term pairs, 16 elements of
             // the head dimension per instruction; both operands K-major (rows of 128 B, 128-byte swizzle).
             constexpr uint32_t idesc = tc::instr_desc(128, NR, 0);
@@ -394,19 +405,19 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
             int step = 0;
             bool ok = true;
             for (int n = 0; ok; ++n) {
-                ok = tc::mbar_wait(bar_bfull, uint32_t(n) & 1u, abortp, 32);
-                if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 47, n, blockIdx.x); *abortp = 1; break; }
+                ok = tc::mbar_wait_warp(bar_bfull, uint32_t(n) & 1u, abortp, 32);
+                if (!ok) { if (lane == 0) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 47, n, blockIdx.x); *abortp = 1; } break; }
                 const ScoreItem si = score_q[n & 3];
                 if (n >= 1) {       // the selection group has moved the previous item's scores out of tensor memory
-                    ok = tc::mbar_wait(bar_sfree, uint32_t(n - 1) & 1u, abortp, 32);
-                    if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 48, n, blockIdx.x); *abortp = 1; break; }
+                    ok = tc::mbar_wait_warp(bar_sfree, uint32_t(n - 1) & 1u, abortp, 32);
+                    if (!ok) { if (lane == 0) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 48, n, blockIdx.x); *abortp = 1; } break; }
                 }
-                if (si.bh < 0) { tc::mbar_arrive(bar_sfull); break; }                   // pass the end marker on
+                if (si.bh < 0) { if (lane == 0) tc::mbar_arrive(bar_sfull); break; }                   // pass the end marker on
                 for (int t = 0; t < ntiles && ok; ++t)
                     for (int kq = 0; kq < 2 * KH; ++kq, ++step) {
                         const int buf = step % AST, kh = kq >> 1;
-                        ok = tc::mbar_wait(bar_afull(buf), uint32_t(step / AST) & 1u, abortp, 32);
-                        if (!ok) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 49, step, blockIdx.x); *abortp = 1; break; }
+                        ok = tc::mbar_wait_warp(bar_afull(buf), uint32_t(step / AST) & 1u, abortp, 32);
+                        if (!ok) { if (lane == 0) { if (!*abortp) set_status(a.hdr, CARNATOR_ERR_DEVICE_TIMEOUT, 49, step, blockIdx.x); *abortp = 1; } break; }
                         tc::tc_fence_after();
                         // The tensor cores add into an fp32 accumulator without guard bits, so a long chain of additions
                         // at the magnitude of the score loses a few bits.  The leading product t1 t1 (the only large one)
@@ -419,18 +430,19 @@ build_fused_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_consta
                         for (int p = 0; p < 6; ++p)
 #pragma unroll
                             for (int kk = 0; kk < 2; ++kk)
-                                tc::mma_ss(p == 0 ? d_big : d_small,
+                                mma_ss_elect(p == 0 ? d_big : d_small,
                                            da0 + uint64_t(((buf * 3 + pa[p]) * L::kBoxA + kk * 32) >> 4),
                                            db0 + uint64_t(((pb[p] * KH + kh) * L::kBoxB + (kq & 1) * 64 + kk * 32) >> 4),
                                            idesc, p == 0 ? ((!big_first || kk > 0) ? 1u : 0u) : ((kq > 0 || p > 1 || kk > 0) ? 1u : 0u));
-                        tc::tc_commit(bar_afree(buf));
+                        tc::tc_commit_el(bar_afree(buf));
                     }
                 if (!ok) break;
-                tc::tc_commit(bar_bfree);
-                tc::tc_commit(bar_sfull);
+                tc::tc_commit_el(bar_bfree);
+                tc::tc_commit_el(bar_sfull);
             }
-            tc::tc_commit(bar_drain2);
+            tc::tc_commit_el(bar_drain2);
             tc::mbar_wait_drain(bar_drain2, 0);
+            __syncwarp();
         }
     } else {
     // ================= selection group =================
